@@ -1,0 +1,148 @@
+/* ahakv.h -- C ABI of the B200 (sm_100a) implementation of AhaKV's eviction step.
+ *
+ * AhaKV (arXiv 2506.03762) evicts KV-cache rows per layer and per head in three
+ * steps: an eviction SCORE from the last r queries against all cached keys
+ * (Section 4.1-4.3), a budgeted SELECTION (Algorithm 1) and the COMPACTION of the
+ * surviving K/V rows (Algorithm 1, generation phase, first line of the loop body).
+ *
+ * Notation: B sequences, Hq query heads, Hkv KV heads, G = Hq/Hkv, d head dim,
+ * n cached tokens, n_total logical tokens seen so far, r observation window,
+ * B_r recent window, Bud = B_r + B_s total budget, n_keep = min(n, Bud).
+ *
+ * Conventions that hold for every entry point unless it says otherwise:
+ *  - Every tensor pointer is DEVICE memory owned by the caller.  The library
+ *    allocates nothing per call; scratch comes from the caller (`ws`).
+ *  - Calls are asynchronous on `stream` and never synchronise.
+ *  - Argument errors are found on the host before any launch and returned as a
+ *    status; nothing aborts, throws or traps.  No output is written in that case.
+ *  - Inputs are row-major with the head dimension contiguous and every row
+ *    16-byte aligned.  Default layout is q_obs [B,Hq,r,d], k and v [B,Hkv,n,d];
+ *    other layouts are described by element strides (batch, head, token).
+ *  - Outputs are dense: score [B,Hkv,n] float32, kept_idx [B,Hkv,n_keep] int32
+ *    strictly ascending per (b, KV head), k_out and v_out [B,Hkv,n_keep,d] in the
+ *    input dtype, score_out [B,Hkv,n_keep] float32.  Outputs must not alias inputs.
+ *  - q_obs holds the queries of the last r positions and k, v the cache, all as
+ *    the attention layer uses them (after any positional rotation).
+ */
+#ifndef AHAKV_H_
+#define AHAKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  AHAKV_OK = 0,
+  AHAKV_ERR_INVALID_ARG = 1, /* a pointer, size, stride or parameter is wrong            */
+  AHAKV_ERR_UNSUPPORTED = 2, /* a legal request this build has no kernel for            */
+  AHAKV_ERR_WORKSPACE = 3,   /* ws is null, misaligned or smaller than required          */
+  AHAKV_ERR_CUDA = 4,        /* a CUDA runtime call or a launch failed                   */
+  AHAKV_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see last_device_status) */
+} ahakv_status;
+
+typedef enum { AHAKV_F32 = 0, AHAKV_F16 = 1, AHAKV_BF16 = 2 } ahakv_dtype;
+
+typedef enum {
+  AHAKV_SCALE_FIXED = 0,         /* lambda = scale for every row; 1/sqrt(d) is the plain softmax of Eq. 1 */
+  AHAKV_SCALE_ADAPTIVE_ROW = 1,  /* Eq. 12 per observation row, i = the row's logical position + 1       */
+  AHAKV_SCALE_ADAPTIVE_CALL = 2  /* Eq. 12 once, with i = n_total                                         */
+} ahakv_scale_mode;
+
+enum {
+  AHAKV_FLAG_VALUE_PRIOR = 1,   /* refine the score with Eq. 13-15                                   */
+  AHAKV_FLAG_POOL_ZERO_PAD = 2, /* Eq. 13's mean filter divides edge windows by the full width        */
+  AHAKV_FLAG_GROUP_MAX = 4      /* pool grouped query heads by max instead of mean (not built yet)    */
+};
+
+typedef struct CUstream_st* ahakv_stream_t; /* a cudaStream_t; NULL is the legacy default stream */
+
+typedef struct {
+  int32_t batch, n_q_heads, n_kv_heads; /* n_q_heads % n_kv_heads == 0                              */
+  int32_t head_dim;                     /* 64 or 128                                                */
+  int32_t n_ctx;                        /* n: rows currently in k and v, >= 1                       */
+  int64_t n_total;                      /* tokens seen so far, >= n_ctx (== n_ctx during prefill)   */
+  int32_t obs_window;                   /* r: 1 .. min(n_ctx, 256 / G)                              */
+  int32_t recent_window;                /* B_r: 0 .. budget                                         */
+  int32_t budget;                       /* Bud >= 1                                                 */
+  int32_t dtype;                        /* ahakv_dtype of q_obs, k, v, k_out, v_out                 */
+  int32_t scale_mode;                   /* ahakv_scale_mode                                         */
+  float scale;                          /* lambda for AHAKV_SCALE_FIXED (> 0)                       */
+  int32_t pool_kernel;                  /* odd width >= 1 of Eq. 13's mean filter; 1 = no smoothing */
+  uint32_t flags;
+  int64_t q_stride[3], k_stride[3], v_stride[3]; /* elements: batch, head, token; all 0 = dense default */
+} ahakv_params;
+
+/* Bytes of scratch the other entry points need for these parameters (0 if they are invalid).
+ * The pointer handed in as `ws` must be 256-byte aligned.  The scratch holds no state between
+ * calls, but two calls that overlap on the GPU must not share it. */
+size_t ahakv_workspace_bytes(const ahakv_params* p);
+
+/* Eq. 12 (Section 4.2): lambda = sqrt(2 ln(n_total / budget) / head_dim), natural log, on the host.
+ * Returns 1/sqrt(head_dim) when n_total <= budget, where Eq. 12 has no real value. */
+double ahakv_lambda(int64_t n_total, int32_t budget, int32_t head_dim);
+
+/* Eviction score (Sections 4.1-4.3; Algorithm 1, Prefill lines 6-10 and Generation line F_t):
+ *   a_ij = SG-softmax over the keys row i may see (Eq. 1 with the causal mask, Eq. 9 with
+ *          lambda from scale_mode, lambda multiplying the raw dot product q.k),
+ *   S_j  = sum of a_ij over the r observation rows (Eq. 5), averaged over the G query heads of
+ *          the KV head,
+ *   with AHAKV_FLAG_VALUE_PRIOR: S_j *= avgpool(|V|^2)_j / max avgpool(|V|^2) (Eq. 13-15),
+ *   with score_prev != NULL: S_j += score_prev_j (Algorithm 1: F_t = ... + F_{t-1}).
+ * Observation row i sits at logical position n_total - r + i and sees cache rows 0 .. n - r + i.
+ * score_prev: nullable, [B,Hkv,n] float32.  score: [B,Hkv,n] float32 out.
+ * v may be NULL when the value prior is off. */
+ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
+                         const float* score_prev, float* score, void* ws, size_t ws_bytes,
+                         ahakv_stream_t stream);
+
+/* Selection (Algorithm 1: S^r = recent B_r tokens, S^s = TopK(F, B_s), S = S^s U S^r).
+ * Keeps rows [n - B_r, n) and the B_s = budget - B_r highest-scoring rows of [0, n - B_r);
+ * equal scores are taken lowest index first; the result is ascending.  n <= budget keeps all rows.
+ * score: [B,Hkv,n] float32 in.  kept_idx: [B,Hkv,n_keep] int32 out. */
+ahakv_status ahakv_select(const ahakv_params* p, const float* score, int32_t* kept_idx, void* ws,
+                          size_t ws_bytes, ahakv_stream_t stream);
+
+/* Compaction (Algorithm 1, Generation: K <- K_S, V <- V_S): row t of the outputs is a byte copy of
+ * row kept_idx[t] of the inputs.  score / score_out are nullable together and gather the score the
+ * same way, so that it can be carried into the next round.  Indices outside [0, n) are an error
+ * the caller must not make: they are not checked on the device. */
+ahakv_status ahakv_compact(const ahakv_params* p, const void* k, const void* v, const float* score,
+                           const int32_t* kept_idx, void* k_out, void* v_out, float* score_out,
+                           ahakv_stream_t stream);
+
+/* The whole step for one layer: score, select, compact, queued back to back on `stream` with no host
+ * synchronisation in between.  score_prev and score_out are nullable; kept_idx is required. */
+ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
+                         const float* score_prev, void* k_out, void* v_out, float* score_out,
+                         int32_t* kept_idx, void* ws, size_t ws_bytes, ahakv_stream_t stream);
+
+/* Reads the status word the kernels of the last call on this workspace left in `ws` (synchronises
+ * `stream`).  AHAKV_OK, or AHAKV_ERR_TIMEOUT if a bounded device-side wait gave up, in which case
+ * the call's outputs are not valid. */
+ahakv_status ahakv_last_device_status(const void* ws, ahakv_stream_t stream);
+
+/* Stage timing, for measurement only (no counterpart in the paper).  While enabled, ahakv_score and
+ * ahakv_evict record CUDA events on the caller's stream around each stage: 0 the scoring kernels
+ * (logits, SG-softmax, column sums), 1 the |V|^2 stream, 2 the value-prior refinement, 3 selection,
+ * 4 compaction.  ahakv_profile_enable(1) creates the events (the only allocation the library ever
+ * makes) and clears the totals; ahakv_profile_enable(0) destroys them.  ahakv_profile_read
+ * synchronises the device, adds up the milliseconds per stage over the calls made since the last
+ * read (at most AHAKV_PROFILE_MAX_CALLS are kept; older ones are dropped), writes them to
+ * ms[AHAKV_N_STAGES] and returns the number of calls covered, or -1 when profiling is off. */
+enum { AHAKV_N_STAGES = 5, AHAKV_PROFILE_MAX_CALLS = 256 };
+ahakv_status ahakv_profile_enable(int on);
+int64_t ahakv_profile_read(double* ms);
+const char* ahakv_stage_name(int stage);
+
+/* Number of kernels the library has launched in this process since it was loaded. */
+int64_t ahakv_launch_count(void);
+
+const char* ahakv_status_string(ahakv_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AHAKV_H_ */

@@ -1,0 +1,236 @@
+"""Thin ctypes binding of libahakv.so: same names as the C ABI, argument marshalling only.
+
+Every step of the eviction path runs in the library's CUDA kernels; PyTorch is
+used here for device memory and streams.  There is no CPU fallback: if the
+shared library is missing, loading fails with an error that says how to build it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass, field
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libahakv.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+F32, F16, BF16 = 0, 1, 2
+SCALE_FIXED, SCALE_ADAPTIVE_ROW, SCALE_ADAPTIVE_CALL = 0, 1, 2
+FLAG_VALUE_PRIOR, FLAG_POOL_ZERO_PAD, FLAG_GROUP_MAX = 1, 2, 4
+
+DTYPE_CODE = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
+CODE_DTYPE = {v: k for k, v in DTYPE_CODE.items()}
+
+
+class AhakvError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class CParams(ctypes.Structure):
+    """Mirror of ``ahakv_params``."""
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("n_ctx", ctypes.c_int32), ("n_total", ctypes.c_int64),
+        ("obs_window", ctypes.c_int32), ("recent_window", ctypes.c_int32), ("budget", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("scale_mode", ctypes.c_int32), ("scale", ctypes.c_float),
+        ("pool_kernel", ctypes.c_int32), ("flags", ctypes.c_uint32),
+        ("q_stride", ctypes.c_int64 * 3), ("k_stride", ctypes.c_int64 * 3), ("v_stride", ctypes.c_int64 * 3),
+    ]
+
+
+@dataclass
+class Params:
+    batch: int
+    n_q_heads: int
+    n_kv_heads: int
+    head_dim: int
+    n_ctx: int
+    obs_window: int
+    recent_window: int
+    budget: int
+    dtype: int = F16
+    n_total: int | None = None           # None: prefill, n_total = n_ctx
+    scale_mode: int = SCALE_ADAPTIVE_ROW
+    scale: float = 0.0
+    pool_kernel: int = 7
+    flags: int = FLAG_VALUE_PRIOR
+    q_stride: tuple = field(default=(0, 0, 0))
+    k_stride: tuple = field(default=(0, 0, 0))
+    v_stride: tuple = field(default=(0, 0, 0))
+
+    def c(self) -> CParams:
+        nt = self.n_ctx if self.n_total is None else self.n_total
+        return CParams(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.n_ctx, nt,
+                       self.obs_window, self.recent_window, self.budget, self.dtype, self.scale_mode,
+                       float(self.scale), self.pool_kernel, self.flags,
+                       (ctypes.c_int64 * 3)(*self.q_stride), (ctypes.c_int64 * 3)(*self.k_stride),
+                       (ctypes.c_int64 * 3)(*self.v_stride))
+
+    @property
+    def n_keep(self) -> int:
+        return min(self.n_ctx, self.budget)
+
+
+_lib = None
+_vp, _sz = ctypes.c_void_p, ctypes.c_size_t
+_PP = ctypes.POINTER(CParams)
+
+SIGNATURES = {
+    "ahakv_workspace_bytes": (_sz, [_PP]),
+    "ahakv_lambda": (ctypes.c_double, [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32]),
+    "ahakv_score": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_select": (ctypes.c_int, [_PP, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_compact": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "ahakv_evict": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_last_device_status": (ctypes.c_int, [_vp, _vp]),
+    "ahakv_launch_count": (ctypes.c_int64, []),
+    "ahakv_profile_enable": (ctypes.c_int, [ctypes.c_int]),
+    "ahakv_profile_read": (ctypes.c_int64, [ctypes.POINTER(ctypes.c_double)]),
+    "ahakv_stage_name": (ctypes.c_char_p, [ctypes.c_int]),
+    "ahakv_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+}
+
+
+def lib():
+    """The loaded C library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2506_03762_b200.build` "
+                "(needs nvcc). This package has no CPU fallback.")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().ahakv_status_string(int(status)).decode()
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _raise(status: int, where: str):
+    if status != OK:
+        raise AhakvError(status, where)
+
+
+def ahakv_workspace_bytes(p: Params) -> int:
+    cp = p.c()
+    return int(lib().ahakv_workspace_bytes(ctypes.byref(cp)))
+
+
+def ahakv_lambda(n_total: int, budget: int, head_dim: int) -> float:
+    return float(lib().ahakv_lambda(n_total, budget, head_dim))
+
+
+def ahakv_launch_count() -> int:
+    return int(lib().ahakv_launch_count())
+
+
+def ahakv_score(p: Params, q_obs, k, v, score_prev, score, ws, ws_bytes: int | None = None, stream=None,
+                check: bool = True) -> int:
+    cp = p.c()
+    nbytes = ws.numel() * ws.element_size() if ws_bytes is None else ws_bytes
+    st = lib().ahakv_score(ctypes.byref(cp), _ptr(q_obs), _ptr(k), _ptr(v), _ptr(score_prev), _ptr(score),
+                           _ptr(ws), nbytes, _stream(stream))
+    if check:
+        _raise(st, "ahakv_score")
+    return st
+
+
+def ahakv_select(p: Params, score, kept_idx, ws, ws_bytes: int | None = None, stream=None,
+                 check: bool = True) -> int:
+    cp = p.c()
+    nbytes = ws.numel() * ws.element_size() if ws_bytes is None else ws_bytes
+    st = lib().ahakv_select(ctypes.byref(cp), _ptr(score), _ptr(kept_idx), _ptr(ws), nbytes, _stream(stream))
+    if check:
+        _raise(st, "ahakv_select")
+    return st
+
+
+def ahakv_compact(p: Params, k, v, score, kept_idx, k_out, v_out, score_out, stream=None,
+                  check: bool = True) -> int:
+    cp = p.c()
+    st = lib().ahakv_compact(ctypes.byref(cp), _ptr(k), _ptr(v), _ptr(score), _ptr(kept_idx), _ptr(k_out),
+                             _ptr(v_out), _ptr(score_out), _stream(stream))
+    if check:
+        _raise(st, "ahakv_compact")
+    return st
+
+
+def ahakv_evict(p: Params, q_obs, k, v, score_prev, k_out, v_out, score_out, kept_idx, ws,
+                ws_bytes: int | None = None, stream=None, check: bool = True) -> int:
+    cp = p.c()
+    nbytes = ws.numel() * ws.element_size() if ws_bytes is None else ws_bytes
+    st = lib().ahakv_evict(ctypes.byref(cp), _ptr(q_obs), _ptr(k), _ptr(v), _ptr(score_prev), _ptr(k_out),
+                           _ptr(v_out), _ptr(score_out), _ptr(kept_idx), _ptr(ws), nbytes, _stream(stream))
+    if check:
+        _raise(st, "ahakv_evict")
+    return st
+
+
+def ahakv_last_device_status(ws, stream=None) -> int:
+    return int(lib().ahakv_last_device_status(_ptr(ws), _stream(stream)))
+
+
+N_STAGES = 5
+
+
+def ahakv_profile_enable(on: bool) -> None:
+    _raise(lib().ahakv_profile_enable(1 if on else 0), "ahakv_profile_enable")
+
+
+def ahakv_profile_read():
+    """(calls, {stage name: total milliseconds}) since the last read; synchronises the device."""
+    ms = (ctypes.c_double * N_STAGES)()
+    calls = int(lib().ahakv_profile_read(ms))
+    return calls, {lib().ahakv_stage_name(t).decode(): ms[t] for t in range(N_STAGES)}
+
+
+# ---- convenience for callers that hold torch tensors -------------------------------------------
+
+def params_for(q_obs: torch.Tensor, k: torch.Tensor, *, recent_window: int, budget: int,
+               n_total: int | None = None, **kw) -> Params:
+    """Params for dense q_obs [B,Hq,r,d] and k [B,Hkv,n,d]."""
+    B, Hq, r, d = q_obs.shape
+    _, Hkv, n, _ = k.shape
+    return Params(B, Hq, Hkv, d, n, r, recent_window, budget, dtype=DTYPE_CODE[k.dtype], n_total=n_total, **kw)
+
+
+def alloc_workspace(p: Params, device="cuda") -> torch.Tensor:
+    nbytes = ahakv_workspace_bytes(p)
+    if nbytes == 0:
+        raise AhakvError(ERR_INVALID_ARG, "ahakv_workspace_bytes")
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
+def alloc_outputs(p: Params, device="cuda"):
+    """(k_out, v_out, score_out, kept_idx) with the shapes the C ABI writes."""
+    dt = CODE_DTYPE[p.dtype]
+    shape = (p.batch, p.n_kv_heads, p.n_keep)
+    return (torch.empty(shape + (p.head_dim,), dtype=dt, device=device),
+            torch.empty(shape + (p.head_dim,), dtype=dt, device=device),
+            torch.empty(shape, dtype=torch.float32, device=device),
+            torch.empty(shape, dtype=torch.int32, device=device))

@@ -1,0 +1,256 @@
+// Host side of libahakv.so: argument checking, the per-call plan, the workspace
+// layout and the order in which the kernels are queued.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+
+#include "ahakv_internal.cuh"
+
+static_assert(sizeof(ahakv_params) == 136, "ahakv_params layout is part of the ABI");
+
+namespace ahakv {
+
+static std::atomic<long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Eq. 12 in double on the host; outside its domain the plain 1/sqrt(d).
+static double eq12(double tokens, double budget, int d) {
+  const double ratio = tokens / budget;
+  if (!(ratio > 1.0)) return 1.0 / std::sqrt((double)d);
+  return std::sqrt(2.0 * std::log(ratio) / (double)d);
+}
+
+static bool resolve_strides(const int64_t in[3], long long out[3], long long heads, long long tokens, int d,
+                            int es) {
+  if (in[0] == 0 && in[1] == 0 && in[2] == 0) {
+    out[2] = d;
+    out[1] = tokens * d;
+    out[0] = heads * tokens * d;
+    return true;
+  }
+  const long long per16 = 16 / es;
+  for (int t = 0; t < 3; ++t) {
+    if (in[t] <= 0 || in[t] % per16 != 0) return false;  // rows must stay 16-byte aligned
+    out[t] = in[t];
+  }
+  return out[2] >= d;
+}
+
+ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
+  if (!p || !pl) return AHAKV_ERR_INVALID_ARG;
+  if (p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_q_heads % p->n_kv_heads != 0)
+    return AHAKV_ERR_INVALID_ARG;
+  if (p->head_dim != 64 && p->head_dim != 128) return AHAKV_ERR_INVALID_ARG;
+  if (p->n_ctx < 1 || p->n_total < p->n_ctx) return AHAKV_ERR_INVALID_ARG;
+  if (p->dtype < AHAKV_F32 || p->dtype > AHAKV_BF16) return AHAKV_ERR_INVALID_ARG;
+  if (p->budget < 1 || p->recent_window < 0 || p->recent_window > p->budget) return AHAKV_ERR_INVALID_ARG;
+  const int G = p->n_q_heads / p->n_kv_heads;
+  if (p->obs_window < 1 || p->obs_window > p->n_ctx || (long long)p->obs_window * G > kMaxRows)
+    return AHAKV_ERR_INVALID_ARG;
+  if (p->scale_mode < AHAKV_SCALE_FIXED || p->scale_mode > AHAKV_SCALE_ADAPTIVE_CALL) return AHAKV_ERR_INVALID_ARG;
+  if (p->scale_mode == AHAKV_SCALE_FIXED && !(p->scale > 0.f && std::isfinite(p->scale)))
+    return AHAKV_ERR_INVALID_ARG;
+  if (p->pool_kernel < 1 || (p->pool_kernel & 1) == 0) return AHAKV_ERR_INVALID_ARG;
+  if (p->flags & ~(uint32_t)(AHAKV_FLAG_VALUE_PRIOR | AHAKV_FLAG_POOL_ZERO_PAD | AHAKV_FLAG_GROUP_MAX))
+    return AHAKV_ERR_INVALID_ARG;
+  if ((long long)p->batch * p->n_kv_heads > 65535LL) return AHAKV_ERR_INVALID_ARG;
+  if (p->flags & AHAKV_FLAG_GROUP_MAX) return AHAKV_ERR_UNSUPPORTED;
+
+  Plan& o = *pl;
+  o.B = p->batch; o.Hq = p->n_q_heads; o.Hkv = p->n_kv_heads; o.G = G; o.d = p->head_dim;
+  o.n = p->n_ctx; o.r = p->obs_window; o.Br = p->recent_window; o.Bud = p->budget;
+  o.Bs = p->budget - p->recent_window;
+  o.n_keep = p->n_ctx < p->budget ? p->n_ctx : p->budget;
+  o.dtype = p->dtype; o.es = p->dtype == AHAKV_F32 ? 4 : 2;
+  o.pool = p->pool_kernel; o.flags = p->flags; o.n_total = p->n_total;
+  o.R = G * p->obs_window;
+  o.n_blk = (o.n + kKeyTile - 1) / kKeyTile;
+  if (!resolve_strides(p->q_stride, o.qs, o.Hq, o.r, o.d, o.es) ||
+      !resolve_strides(p->k_stride, o.ks, o.Hkv, o.n, o.d, o.es) ||
+      !resolve_strides(p->v_stride, o.vs, o.Hkv, o.n, o.d, o.es))
+    return AHAKV_ERR_INVALID_ARG;
+
+  for (int i = 0; i < kMaxRows; ++i) o.rows.c[i] = 0.f;
+  for (int i = 0; i < o.r; ++i) {
+    double lam;
+    if (p->scale_mode == AHAKV_SCALE_FIXED) lam = (double)p->scale;
+    else if (p->scale_mode == AHAKV_SCALE_ADAPTIVE_ROW)
+      lam = eq12((double)(p->n_total - p->obs_window + i + 1), (double)p->budget, p->head_dim);
+    else lam = eq12((double)p->n_total, (double)p->budget, p->head_dim);
+    o.rows.c[i] = (float)(lam * 1.4426950408889634);
+  }
+
+  // Tensor-core scoring: 16-bit inputs; query heads of a row block must form one TMA box.
+  o.heads_per_rb = 1; o.n_rb = 1; o.use_tc = false;
+  if (o.es == 2 && score_tc_available()) {
+    if (o.r <= 128) {
+      int hb = 128 / o.r;
+      if (hb > G) hb = G;
+      o.heads_per_rb = hb;
+      o.n_rb = (G + hb - 1) / hb;
+      o.use_tc = (G % hb == 0);
+    } else {              // one query head split over two row blocks
+      o.heads_per_rb = 1;
+      o.n_rb = 2;
+      o.use_tc = (G == 1);
+    }
+  }
+  const int rb_slots = o.use_tc ? o.n_rb : 1;
+
+  const size_t units = (size_t)o.B * o.Hkv;
+  size_t off = 0;
+  o.off_status = off;  off += 256;
+  o.off_sync = off;    off += align_up(units * rb_slots * 2 * sizeof(int), 256);
+  o.off_sraw = off;    off += align_up(units * rb_slots * o.n * sizeof(float), 256);
+  o.off_nu = off;      off += align_up(units * o.n * sizeof(float), 256);
+  o.off_partial = off; off += align_up(units * rb_slots * o.n_blk * (o.use_tc ? 128 : o.R) * sizeof(float2), 256);
+  o.off_final = off;   off += align_up(units * rb_slots * (o.use_tc ? 128 : o.R) * sizeof(float2), 256);
+  o.off_score = off;   off += align_up(units * o.n * sizeof(float), 256);
+  o.ws_total = off;
+  return AHAKV_OK;
+}
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+static ahakv_status check_ws(const Plan& pl, void* ws, size_t ws_bytes) {
+  if (!ws || ((uintptr_t)ws & 255) != 0 || ws_bytes < pl.ws_total) return AHAKV_ERR_WORKSPACE;
+  return AHAKV_OK;
+}
+
+template <typename T> static T* at(void* ws, size_t off) { return reinterpret_cast<T*>((char*)ws + off); }
+
+// Queues the scoring kernels; the refined score lands in `score`.
+static ahakv_status queue_score(const Plan& pl, const void* q, const void* k, const void* v,
+                                const float* score_prev, float* score, void* ws, cudaStream_t st, int prof) {
+  ahakv_status rc = cuda_ok(cudaMemsetAsync(at<char>(ws, pl.off_status), 0, pl.off_sraw - pl.off_status, st));
+  if (rc) return rc;
+  profile_mark(prof, 0, st);
+  float* s_raw = at<float>(ws, pl.off_sraw);
+  float2* partial = at<float2>(ws, pl.off_partial);
+  float* final_off = at<float>(ws, pl.off_final);
+  if (pl.use_tc)
+    rc = launch_score_tc(pl, q, k, s_raw, partial, final_off, at<int>(ws, pl.off_sync),
+                         at<int>(ws, pl.off_status), st);
+  else
+    rc = launch_score_simt(pl, q, k, s_raw, partial, final_off, st);
+  if (rc) return rc;
+  profile_mark(prof, 1, st);
+  float* nu = nullptr;
+  if (pl.flags & AHAKV_FLAG_VALUE_PRIOR) {
+    nu = at<float>(ws, pl.off_nu);
+    rc = launch_vnorm(pl, v, nu, st);
+    if (rc) return rc;
+  }
+  profile_mark(prof, 2, st);
+  rc = launch_refine(pl, s_raw, nu, score_prev, score, st);
+  profile_mark(prof, 3, st);
+  return rc;
+}
+
+}  // namespace ahakv
+
+using namespace ahakv;
+
+extern "C" {
+
+size_t ahakv_workspace_bytes(const ahakv_params* p) {
+  Plan pl;
+  if (make_plan(p, &pl) != AHAKV_OK) return 0;
+  return pl.ws_total;
+}
+
+double ahakv_lambda(int64_t n_total, int32_t budget, int32_t head_dim) {
+  if (budget < 1 || head_dim < 1) return 0.0;
+  return eq12((double)n_total, (double)budget, head_dim);
+}
+
+ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
+                         const float* score_prev, float* score, void* ws, size_t ws_bytes,
+                         ahakv_stream_t stream) {
+  Plan pl;
+  ahakv_status rc = make_plan(p, &pl);
+  if (rc) return rc;
+  const bool prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0;
+  if (!q_obs || !k || !score || (prior && !v)) return AHAKV_ERR_INVALID_ARG;
+  if (!aligned16(q_obs) || !aligned16(k) || (v && !aligned16(v)) || !aligned16(score) ||
+      (score_prev && !aligned16(score_prev)))
+    return AHAKV_ERR_INVALID_ARG;
+  if ((rc = check_ws(pl, ws, ws_bytes))) return rc;
+  const int prof = profile_begin_call((cudaStream_t)stream);
+  rc = queue_score(pl, q_obs, k, v, score_prev, score, ws, (cudaStream_t)stream, prof);
+  profile_mark(prof, 4, (cudaStream_t)stream);   // no selection or compaction in this call
+  profile_mark(prof, 5, (cudaStream_t)stream);
+  return rc;
+}
+
+ahakv_status ahakv_select(const ahakv_params* p, const float* score, int32_t* kept_idx, void* ws,
+                          size_t ws_bytes, ahakv_stream_t stream) {
+  Plan pl;
+  ahakv_status rc = make_plan(p, &pl);
+  if (rc) return rc;
+  if (!score || !kept_idx || !aligned16(score) || ((uintptr_t)kept_idx & 3)) return AHAKV_ERR_INVALID_ARG;
+  if ((rc = check_ws(pl, ws, ws_bytes))) return rc;
+  return launch_select(pl, score, kept_idx, (cudaStream_t)stream);
+}
+
+ahakv_status ahakv_compact(const ahakv_params* p, const void* k, const void* v, const float* score,
+                           const int32_t* kept_idx, void* k_out, void* v_out, float* score_out,
+                           ahakv_stream_t stream) {
+  Plan pl;
+  ahakv_status rc = make_plan(p, &pl);
+  if (rc) return rc;
+  if (!k || !v || !kept_idx || !k_out || !v_out) return AHAKV_ERR_INVALID_ARG;
+  if ((score == nullptr) != (score_out == nullptr)) return AHAKV_ERR_INVALID_ARG;
+  if (!aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out) || ((uintptr_t)kept_idx & 3))
+    return AHAKV_ERR_INVALID_ARG;
+  return launch_compact(pl, k, v, score, kept_idx, k_out, v_out, score_out, (cudaStream_t)stream);
+}
+
+ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
+                         const float* score_prev, void* k_out, void* v_out, float* score_out,
+                         int32_t* kept_idx, void* ws, size_t ws_bytes, ahakv_stream_t stream) {
+  Plan pl;
+  ahakv_status rc = make_plan(p, &pl);
+  if (rc) return rc;
+  if (!q_obs || !k || !v || !k_out || !v_out || !kept_idx) return AHAKV_ERR_INVALID_ARG;
+  if (!aligned16(q_obs) || !aligned16(k) || !aligned16(v) || !aligned16(k_out) || !aligned16(v_out) ||
+      ((uintptr_t)kept_idx & 3) || (score_prev && !aligned16(score_prev)))
+    return AHAKV_ERR_INVALID_ARG;
+  if ((rc = check_ws(pl, ws, ws_bytes))) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  float* score = at<float>(ws, pl.off_score);
+  const int prof = profile_begin_call(st);
+  if ((rc = queue_score(pl, q_obs, k, v, score_prev, score, ws, st, prof))) return rc;
+  if ((rc = launch_select(pl, score, kept_idx, st))) return rc;
+  profile_mark(prof, 4, st);
+  rc = launch_compact(pl, k, v, score_out ? score : nullptr, kept_idx, k_out, v_out, score_out, st);
+  profile_mark(prof, 5, st);
+  return rc;
+}
+
+ahakv_status ahakv_last_device_status(const void* ws, ahakv_stream_t stream) {
+  if (!ws) return AHAKV_ERR_WORKSPACE;
+  int word = 0;
+  if (cudaMemcpyAsync(&word, ws, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess)
+    return AHAKV_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return AHAKV_ERR_CUDA;
+  return word == 0 ? AHAKV_OK : AHAKV_ERR_TIMEOUT;
+}
+
+int64_t ahakv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* ahakv_status_string(ahakv_status s) {
+  switch (s) {
+    case AHAKV_OK: return "ok";
+    case AHAKV_ERR_INVALID_ARG: return "invalid argument";
+    case AHAKV_ERR_UNSUPPORTED: return "unsupported request";
+    case AHAKV_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case AHAKV_ERR_CUDA: return "CUDA call or launch failed";
+    case AHAKV_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"
