@@ -84,7 +84,7 @@ ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
 
   // Tensor-core scoring: 16-bit inputs; query heads of a row block must form one TMA box.
   o.heads_per_rb = 1; o.n_rb = 1; o.use_tc = false;
-  if (o.es == 2 && score_tc_available()) {
+  if (o.es == 2 && o.n >= kKeyTile && (long long)o.B * o.Hkv * 2 * o.n_blk < (1LL << 30) && score_tc_available()) {
     if (o.r <= 128) {
       int hb = 128 / o.r;
       if (hb > G) hb = G;
