@@ -36,6 +36,9 @@ def parse_args():
                     help="distinct layers of input kept in HBM and cycled through")
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling small cases)")
+    ap.add_argument("--capture", action="store_true",
+                    help="profiler-friendly run: exactly --warmup and --steps calls of ahakv_evict, nothing else")
     return ap.parse_args()
 
 
@@ -197,6 +200,8 @@ def run_ours(args):
     ab.lib()
 
     w = synth.WORKLOADS[args.workload]
+    if args.batch > 0:
+        w = w.scaled(batch=args.batch)
     flags = ab.FLAG_VALUE_PRIOR if w.value_prior else 0
     p = ab.Params(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.n_ctx, w.obs_window, w.recent_window,
                   w.budget, dtype={"f32": ab.F32, "f16": ab.F16, "bf16": ab.BF16}[w.dtype],
@@ -217,9 +222,17 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(max(args.warmup, 3)):
+    n_warm = args.warmup if args.capture else max(args.warmup, 3)
+    for i in range(n_warm):
         step(i)
     barrier()
+    if args.capture:
+        for i in range(args.steps):
+            step(i)
+        barrier()
+        print(json.dumps({"capture": True, "workload": w.name, "batch": w.batch, "steps": args.steps,
+                          "warmup": n_warm, "device_status": ab.ahakv_last_device_status(ws)}))
+        return
     assert ab.ahakv_last_device_status(ws) == ab.OK, "device-side wait timed out during warm-up"
 
     # ---- timed region: exactly K steps, device-timed -------------------------------------------------
@@ -307,7 +320,7 @@ def run_ours(args):
                 "slowest_stage": top}
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": n_warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": workload_config(w, args),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": int(status),
         "roofline": roofline,

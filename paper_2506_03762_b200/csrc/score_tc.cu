@@ -34,18 +34,19 @@ namespace {
 
 constexpr int kStages = 2;                 // K-tile ring depth per pipeline
 constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 16-bit elements, 128-byte swizzled
-constexpr int kThreads = 384;              // 4 service warps + two 4-warp softmax groups
+constexpr int kThreads = 512;              // 4 service warps + two softmax groups + the publisher group
 constexpr long long kWaitLimitNs = 1000000000LL;   // 1 s
 
 struct TcArgs {
   int n, r, G, Hkv, n_rb, hb, n_blk, D;
-  int T;          // tiles = units * n_blk
-  int CH;         // consecutive tiles per run
-  int n_runs;
+  int CH;         // key tiles per run
+  int rpu;        // runs per row block = ceil(n_blk / CH)
+  int n_runs;     // row blocks * rpu
+  int lag;        // pass 1 may lead this CTA's pass 2 by at most this many row blocks
   int bf16;       // operand type of the products
   float log2G;
   float c[kMaxRows];
-  float2* partial;   // [unit][blk][128]
+  float2* partial;   // [unit][run][128]
   float* final_off;  // [unit][128]
   float* s_raw;      // [unit][n]
   int* cnt;          // [unit] partials delivered
@@ -60,12 +61,25 @@ struct __align__(8) Barriers {
   unsigned long long k_empty[2][kStages];
   unsigned long long acc_full[2][2];
   unsigned long long acc_empty[2][2];
+  unsigned long long pub_full[2];          // row statistics of a run: softmax group -> publisher
+  unsigned long long pub_free[2];
+};
+
+struct Shared {
+  Barriers bars;
+  uint32_t tmem_slot;
+  int bcast;
+  int p2_unit;                  // row block pass 2 of this CTA is working on
+  int p2_ready;
+  float c[kMaxRows];            // lambda_i * log2(e) per observation row
+  float2 row_const[128];        // pass 2: (c, offset) per stacked row of the current row block
+  float2 pub[2][128];           // pass 1 -> publisher
 };
 
 constexpr int kQBytes = 2 * kSubTileBytes;              // per pipeline, D <= 128
 constexpr int kKRingBytes = kStages * 2 * kSubTileBytes;
 constexpr int kSmemTiles = 2 * (kQBytes + kKRingBytes);  // 192 KiB
-constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 4096 /*barriers, constants*/;
+constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 8192 /*barriers, constants*/;
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -157,22 +171,29 @@ __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t b
       : "memory");
 }
 
-// 32 consecutive FP32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
-  uint32_t r[32];
+// 32 consecutive FP32 columns of this thread's TMEM lane: issue now, use after tmem_ld_wait(r).
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"      // one statement: no use of the registers can move above the wait
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
-#pragma unroll
-  for (int t = 0; t < 32; ++t) v[t] = __uint_as_float(r[t]);
+}
+// Waits for every TMEM load this thread has issued.  The registers pass through the statement, so no
+// use of them can be scheduled above the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t* r) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
 }
 
 // 16 consecutive FP32 columns of this thread's TMEM lane.
@@ -198,22 +219,20 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
   return v;
 }
 
-// ---- the sequence of tiles one CTA walks (the same in every role) ----------------------------------
-struct TileWalk {
-  int run, t, t_end, T, CH, step;
-  __device__ TileWalk(const TcArgs& a) : run(blockIdx.x), T(a.T), CH(a.CH), step(gridDim.x) { open(); }
-  __device__ void open() {
-    t = run * CH;
-    t_end = min(t + CH, T);
-  }
-  __device__ bool valid() const { return t < T; }
-  __device__ void next() {
-    if (++t >= t_end) {
-      run += step;
-      open();
-    }
-  }
+// ---- work decomposition ----------------------------------------------------------------------------------
+// A run = up to CH consecutive key tiles of one row block.  Run `q` belongs to CTA q % gridDim.x; every role
+// of a CTA walks the same runs in the same order.
+struct Run {
+  int unit, rin, blk0, cnt;
 };
+__device__ __forceinline__ Run run_info(const TcArgs& a, int run) {
+  Run r;
+  r.unit = run / a.rpu;
+  r.rin = run % a.rpu;
+  r.blk0 = r.rin * a.CH;
+  r.cnt = min(a.CH, a.n_blk - r.blk0);
+  return r;
+}
 
 struct UnitInfo {
   int unit, bh, rb, b, h, rows, npad;
@@ -235,222 +254,319 @@ __device__ __forceinline__ int obs_row(const TcArgs& a, const UnitInfo& u, int s
 }
 
 // ---- roles --------------------------------------------------------------------------------------------
-// TMA producer of one pipeline.
-__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, Barriers* bars, int pipe,
+// TMA producer of one pipeline.  The pass-1 producer also keeps pass 1 from running more than `lag` row
+// blocks ahead of this CTA's pass 2, so that the keys pass 2 re-reads are still in L2.
+__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, Shared* sh, int pipe,
                          char* q_smem, char* k_ring) {
+  Barriers* bars = &sh->bars;
   const int n_sub = a.D / 64;
   const int q_rows = a.r <= 128 ? a.hb * a.r : 128;
   const int q_bytes = n_sub * q_rows * 128, k_bytes = n_sub * kSubTileBytes;
-  int it = 0, prev_unit = -1, q_loads = 0;
+  int it = 0, prev_unit = -1;
   bool ok = true;
-  for (TileWalk w(a); w.valid() && ok; w.next(), ++it) {
-    const int unit = w.t / a.n_blk, blk = w.t % a.n_blk;
-    const int stage = it % kStages, ph = (it / kStages) & 1;
-    if (unit != prev_unit) {
+  for (int run = blockIdx.x; run < a.n_runs && ok; run += gridDim.x) {
+    const Run rn = run_info(a, run);
+    const UnitInfo u = unit_info(a, rn.unit);
+    if (pipe == 0 && rn.unit > *(volatile int*)&sh->p2_unit + a.lag) {
+      const long long t0 = now_ns();
+      while (rn.unit > *(volatile int*)&sh->p2_unit + a.lag) {
+        __nanosleep(100);
+        if (now_ns() - t0 > kWaitLimitNs) {
+          atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
+          ok = false;
+          break;
+        }
+      }
+      if (!ok) break;
+    }
+    if (rn.unit != prev_unit) {
       // the Q buffer is free once every product issued so far has completed
       if (it > 0) ok = mbar_wait(&bars->k_empty[pipe][(it - 1) % kStages], ((it - 1) / kStages) & 1, a.status);
       if (!ok) break;
-      const UnitInfo u = unit_info(a, unit);
       mbar_expect_tx(&bars->q_full[pipe], q_bytes);
       for (int s = 0; s < n_sub; ++s) {
         if (a.r <= 128) tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[pipe], s * 64, 0, u.h * a.G + u.rb * a.hb, u.b);
         else tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[pipe], s * 64, u.rb * 128, u.h, u.b);
       }
-      ++q_loads;
-      prev_unit = unit;
+      prev_unit = rn.unit;
     }
-    ok = mbar_wait(&bars->k_empty[pipe][stage], ph ^ 1, a.status);
-    if (!ok) break;
-    const UnitInfo u = unit_info(a, unit);
-    mbar_expect_tx(&bars->k_full[pipe][stage], k_bytes);
-    for (int s = 0; s < n_sub; ++s)
-      tma_load_4d(k_ring + (stage * 2 + s) * kSubTileBytes, kmap, &bars->k_full[pipe][stage], s * 64, blk * kKeyTile,
-                  u.h, u.b);
+    for (int t = 0; t < rn.cnt && ok; ++t, ++it) {
+      const int stage = it % kStages, ph = (it / kStages) & 1;
+      ok = mbar_wait(&bars->k_empty[pipe][stage], ph ^ 1, a.status);
+      if (!ok) break;
+      mbar_expect_tx(&bars->k_full[pipe][stage], k_bytes);
+      for (int s = 0; s < n_sub; ++s)
+        tma_load_4d(k_ring + (stage * 2 + s) * kSubTileBytes, kmap, &bars->k_full[pipe][stage], s * 64,
+                    (rn.blk0 + t) * kKeyTile, u.h, u.b);
+    }
   }
   if (!ok) {
     // wind down: give copies already in flight a bounded time (1 ms) to land before the CTA exits
     const long long t0 = now_ns();
     while (now_ns() - t0 < 1000000) __nanosleep(1000);
   }
-  (void)q_loads;
 }
 
 // MMA issuer of one pipeline.  pipe 0: D[rows x keys] = Q K^T.  pipe 1: D[keys x rows] = K Q^T.
-__device__ void mma_issuer(const TcArgs& a, Barriers* bars, int pipe, char* q_smem, char* k_ring, uint32_t tmem_base) {
-  const int n_sub = a.D / 64;
+__device__ void mma_issuer(const TcArgs& a, Shared* sh, int pipe, char* q_smem, char* k_ring, uint32_t tmem_base) {
+  Barriers* bars = &sh->bars;
   int it = 0, prev_unit = -1, q_loads = 0;
   uint32_t idesc = umma_idesc(128, 128, a.bf16);
-  for (TileWalk w(a); w.valid(); w.next(), ++it) {
-    const int unit = w.t / a.n_blk;
-    const int stage = it % kStages, ph = (it / kStages) & 1, acc = it & 1, aph = (it >> 1) & 1;
-    if (unit != prev_unit) {
+  for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x) {
+    const Run rn = run_info(a, run);
+    if (rn.unit != prev_unit) {
       if (!mbar_wait(&bars->q_full[pipe], q_loads & 1, a.status)) return;
       ++q_loads;
-      prev_unit = unit;
-      if (pipe == 1) idesc = umma_idesc(128, unit_info(a, unit).npad, a.bf16);
+      prev_unit = rn.unit;
+      if (pipe == 1) idesc = umma_idesc(128, unit_info(a, rn.unit).npad, a.bf16);
     }
-    if (!mbar_wait(&bars->acc_empty[pipe][acc], aph ^ 1, a.status)) return;
-    if (!mbar_wait(&bars->k_full[pipe][stage], ph, a.status)) return;
-    tc_fence_after();
-    const uint32_t d_tmem = tmem_base + (uint32_t)((pipe * 2 + acc) * 128);
-    for (int kk = 0; kk < a.D / 16; ++kk) {
-      const int sub = kk >> 2, koff = (kk & 3) * 32;
-      const uint64_t qd = umma_desc(smem_u32(q_smem + sub * kSubTileBytes) + koff);
-      const uint64_t kd = umma_desc(smem_u32(k_ring + (stage * 2 + sub) * kSubTileBytes) + koff);
-      if (pipe == 0) umma(d_tmem, qd, kd, idesc, kk > 0);
-      else umma(d_tmem, kd, qd, idesc, kk > 0);
+    for (int t = 0; t < rn.cnt; ++t, ++it) {
+      const int stage = it % kStages, ph = (it / kStages) & 1, acc = it & 1, aph = (it >> 1) & 1;
+      if (!mbar_wait(&bars->acc_empty[pipe][acc], aph ^ 1, a.status)) return;
+      if (!mbar_wait(&bars->k_full[pipe][stage], ph, a.status)) return;
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)((pipe * 2 + acc) * 128);
+      for (int kk = 0; kk < a.D / 16; ++kk) {
+        const int sub = kk >> 2, koff = (kk & 3) * 32;
+        const uint64_t qd = umma_desc(smem_u32(q_smem + sub * kSubTileBytes) + koff);
+        const uint64_t kd = umma_desc(smem_u32(k_ring + (stage * 2 + sub) * kSubTileBytes) + koff);
+        if (pipe == 0) umma(d_tmem, qd, kd, idesc, kk > 0);
+        else umma(d_tmem, kd, qd, idesc, kk > 0);
+      }
+      tc_commit(&bars->k_empty[pipe][stage]);
+      tc_commit(&bars->acc_full[pipe][acc]);
     }
-    tc_commit(&bars->k_empty[pipe][stage]);
-    tc_commit(&bars->acc_full[pipe][acc]);
   }
-  (void)n_sub;
 }
 
-// Pass-1 softmax group: thread `s` owns stacked row s.
-__device__ void row_stats_group(const TcArgs& a, Barriers* bars, uint32_t tmem_base, const float* c_smem, int* bcast) {
-  const int s = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
-  int it = 0;
-  bool dead = false;   // a wait ran out: stay in the group's barrier protocol, skip everything else
-  for (TileWalk w(a); w.valid(); w.next(), ++it) {
-    const int unit = w.t / a.n_blk, blk = w.t % a.n_blk;
-    const UnitInfo u = unit_info(a, unit);
-    const int acc = it & 1, aph = (it >> 1) & 1;
-    if (!dead && !mbar_wait(&bars->acc_full[0][acc], aph, a.status)) dead = true;
-    if (dead) {          // the three barriers of a live iteration, nothing else
-      group_sync(1);
-      if (s == 0) bcast[0] = -1;
-      group_sync(1);
-      group_sync(1);
-      continue;
+// One 32-key chunk of a row: fold (max, sum of 2^{c w - max}) into the running pair.
+__device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_first, int last, float c, float& M,
+                                           float& Z) {
+  float v[32];
+#pragma unroll
+  for (int t = 0; t < 32; ++t) v[t] = __uint_as_float(r[t]);
+  if (!full) {
+#pragma unroll
+    for (int t = 0; t < 32; ++t)
+      if (j_first + t > last) v[t] = -INFINITY;
+  }
+  float mx0 = fmaxf(v[0], v[1]), mx1 = fmaxf(v[2], v[3]);
+#pragma unroll
+  for (int t = 4; t < 32; t += 4) {
+    mx0 = fmaxf(mx0, fmaxf(v[t], v[t + 1]));
+    mx1 = fmaxf(mx1, fmaxf(v[t + 2], v[t + 3]));
+  }
+  const float mx = fmaxf(mx0, mx1);
+  if (mx > -INFINITY) {
+    const float m2 = fmaxf(mx * c, M);          // the running maximum after this chunk
+    const float neg = -m2;
+    float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+#pragma unroll
+    for (int t = 0; t < 32; t += 4) {
+      z0 += fast_exp2(fmaf(v[t], c, neg));
+      z1 += fast_exp2(fmaf(v[t + 1], c, neg));
+      z2 += fast_exp2(fmaf(v[t + 2], c, neg));
+      z3 += fast_exp2(fmaf(v[t + 3], c, neg));
     }
-    tc_fence_after();
+    if (m2 > M) Z *= fast_exp2(M - m2);          // rare once the maximum has settled
+    Z += (z0 + z1) + (z2 + z3);
+    M = m2;
+  }
+}
+
+// Pass-1 softmax group: thread `s` owns stacked row s.  One (max, sum) pair per run goes to the
+// publisher group through shared memory, so this group never waits on global memory.
+__device__ void row_stats_group(const TcArgs& a, Shared* sh, uint32_t tmem_base) {
+  Barriers* bars = &sh->bars;
+  const int s = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
+  int it = 0, run_it = 0;
+  bool dead = false;   // a wait ran out: skip everything that is left
+  for (int run = blockIdx.x; run < a.n_runs && !dead; run += gridDim.x, ++run_it) {
+    const Run rn = run_info(a, run);
+    const UnitInfo u = unit_info(a, rn.unit);
     const int i = obs_row(a, u, s);
-    const float c = c_smem[i < a.r ? i : 0];
-    const int last = a.n - a.r + i;                     // last visible key of this row
-    const int j0 = blk * kKeyTile;
-    const bool full = j0 + kKeyTile - 1 <= a.n - a.r;   // every key of the tile is visible to every row
-    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 128);
+    const float c = sh->c[i < a.r ? i : 0];
+    const int last = a.n - a.r + i;                       // last visible key of this row
     float M = -INFINITY, Z = 0.f;
-#pragma unroll 1
-    for (int ch = 0; ch < 4; ++ch) {
-      float v[32];
-      tmem_ld32(taddr + ch * 32, v);
-      if (!full) {
+    for (int t = 0; t < rn.cnt; ++t, ++it) {
+      const int acc = it & 1, aph = (it >> 1) & 1;
+      if (!mbar_wait(&bars->acc_full[0][acc], aph, a.status)) { dead = true; break; }
+      tc_fence_after();
+      const int j0 = (rn.blk0 + t) * kKeyTile;
+      const bool full = j0 + kKeyTile - 1 <= a.n - a.r;   // every key of the tile is visible to every row
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 128);
+      uint32_t ra[32], rb[32];
+      tmem_ld32_issue(taddr, ra);
+      tmem_ld_wait(ra);
+      tmem_ld32_issue(taddr + 32, rb);
+      fold_chunk(ra, full, j0, last, c, M, Z);
+      tmem_ld_wait(rb);
+      tmem_ld32_issue(taddr + 64, ra);
+      fold_chunk(rb, full, j0 + 32, last, c, M, Z);
+      tmem_ld_wait(ra);
+      tmem_ld32_issue(taddr + 96, rb);
+      fold_chunk(ra, full, j0 + 64, last, c, M, Z);
+      tmem_ld_wait(rb);
+      tc_fence_before();
+      mbar_arrive(&bars->acc_empty[0][acc]);               // the accumulator is free for the next product
+      fold_chunk(rb, full, j0 + 96, last, c, M, Z);
+    }
+    if (dead) break;
+    const int slot = run_it & 1, sph = (run_it >> 1) & 1;
+    if (!mbar_wait(&bars->pub_free[slot], sph ^ 1, a.status)) break;
+    sh->pub[slot][s] = make_float2(M, Z);
+    mbar_arrive(&bars->pub_full[slot]);
+  }
+}
+
+// Publisher group: moves each run's row statistics to global memory, counts the runs of a row block and,
+// on delivering the last one, merges all of them into one offset per row and raises the block's flag.
+__device__ void publisher_group(const TcArgs& a, Shared* sh) {
+  Barriers* bars = &sh->bars;
+  const int s = threadIdx.x & 127;
+  int run_it = 0;
+  bool dead = false;   // a wait ran out: stay in the group's barrier protocol, skip everything else
+  for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x, ++run_it) {
+    const Run rn = run_info(a, run);
+    const int slot = run_it & 1, sph = (run_it >> 1) & 1;
+    if (!dead && !mbar_wait(&bars->pub_full[slot], sph, a.status)) dead = true;
+    if (!dead) {
+      const float2 e = sh->pub[slot][s];
+      mbar_arrive(&bars->pub_free[slot]);
+      a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s] = e;
+      __threadfence();
+    }
+    group_sync(3);
+    if (s == 0) sh->bcast = dead ? -1 : atomicAdd(&a.cnt[rn.unit], 1);
+    group_sync(3);
+    const bool last_run = sh->bcast == a.rpu - 1;
+    group_sync(3);                                         // bcast may be rewritten after this point
+    if (last_run && !dead) {
+      __threadfence();
+      const float2* p = a.partial + (size_t)rn.unit * a.rpu * 128 + s;
+      float Mx = -INFINITY, Zs = 0.f;
+      for (int t0 = 0; t0 < a.rpu; t0 += 16) {             // 16 loads in flight per thread
+        float2 e[16];
 #pragma unroll
-        for (int t = 0; t < 32; ++t)
-          if (j0 + ch * 32 + t > last) v[t] = -INFINITY;
-      }
-      float mx = v[0];
+        for (int t = 0; t < 16; ++t)
+          e[t] = t0 + t < a.rpu ? __ldcg(&p[(size_t)(t0 + t) * 128]) : make_float2(-INFINITY, 0.f);
+        float m = Mx;
 #pragma unroll
-      for (int t = 1; t < 32; ++t) mx = fmaxf(mx, v[t]);
-      if (mx > -INFINITY) {
-        const float m2 = mx * c;
-        float z = 0.f;
+        for (int t = 0; t < 16; ++t) m = fmaxf(m, e[t].x);
+        if (m > -INFINITY) {
+          float z = Zs > 0.f ? Zs * fast_exp2(Mx - m) : 0.f;
 #pragma unroll
-        for (int t = 0; t < 32; ++t) z += fast_exp2(fmaf(v[t], c, -m2));
-        if (m2 > M) {
-          Z = Z * fast_exp2(M - m2) + z;
-          M = m2;
-        } else {
-          Z += z * fast_exp2(m2 - M);
+          for (int t = 0; t < 16; ++t)
+            if (e[t].y > 0.f) z += e[t].y * fast_exp2(e[t].x - m);
+          Zs = z;
+          Mx = m;
         }
       }
-    }
-    tc_fence_before();
-    mbar_arrive(&bars->acc_empty[0][acc]);
-    a.partial[((size_t)unit * a.n_blk + blk) * 128 + s] = make_float2(M, Z);
-    __threadfence();
-    group_sync(1);
-    if (s == 0) bcast[0] = atomicAdd(&a.cnt[unit], 1);   // (a dead thread 0 has written -1 instead)
-    group_sync(1);
-    const bool last_partial = bcast[0] == a.n_blk - 1;
-    group_sync(1);                                       // bcast may be rewritten after this point
-    if (last_partial) {
-      // this CTA delivered the row block's last tile: merge all partials of row s
-      __threadfence();
-      const float2* p = a.partial + (size_t)unit * a.n_blk * 128 + s;
-      float Mx = -INFINITY;
-      for (int t = 0; t < a.n_blk; ++t) Mx = fmaxf(Mx, __ldcg(&p[(size_t)t * 128]).x);
-      float Zs = 0.f;
-      for (int t = 0; t < a.n_blk; ++t) {
-        const float2 e = __ldcg(&p[(size_t)t * 128]);
-        if (e.y > 0.f) Zs += e.y * fast_exp2(e.x - Mx);
-      }
       // 2^{c w - off} = softmax weight / G
-      a.final_off[(size_t)unit * 128 + s] = Mx + log2f(Zs) + a.log2G;
+      a.final_off[(size_t)rn.unit * 128 + s] = Mx + log2f(Zs) + a.log2G;
       __threadfence();
-      atomicAdd(&a.flag[unit], 1);       // the block is ready when all 128 rows have reported
+      atomicAdd(&a.flag[rn.unit], 1);                      // the block is ready when all 128 rows have reported
     }
   }
+}
+
+// One 32-row chunk of a key's column: add 2^{c w - off} over rows [s0, s0 + cols).
+__device__ __forceinline__ float column_chunk(const uint32_t* r, const float4* rc2, int s0, int cols) {
+  float z0 = 0.f, z1 = 0.f;
+#pragma unroll
+  for (int t = 0; t < 32; t += 2) {
+    if (t < 16 || cols > 16) {
+      const float4 k = rc2[(s0 + t) >> 1];                 // (c, off) of two consecutive rows
+      z0 += fast_exp2(fmaf(__uint_as_float(r[t]), k.x, -k.y));
+      z1 += fast_exp2(fmaf(__uint_as_float(r[t + 1]), k.z, -k.w));
+    }
+  }
+  return z0 + z1;
 }
 
 // Pass-2 softmax group: thread `jl` owns key j0 + jl.
-__device__ void column_sum_group(const TcArgs& a, Barriers* bars, uint32_t tmem_base, const float* c_smem,
-                                 float2* row_const) {
+__device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base) {
+  Barriers* bars = &sh->bars;
   const int jl = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
+  const float4* rc2 = reinterpret_cast<const float4*>(sh->row_const);
   int it = 0, prev_unit = -1;
   bool dead = false;     // a flag wait ran out: keep the pipeline protocol, skip the arithmetic
   bool gone = false;     // an accumulator wait ran out: keep only the group barriers
   UnitInfo u = unit_info(a, 0);
-  for (TileWalk w(a); w.valid(); w.next(), ++it) {
-    const int unit = w.t / a.n_blk, blk = w.t % a.n_blk;
-    if (unit != prev_unit) {
-      prev_unit = unit;
-      u = unit_info(a, unit);
-      if (!dead) {
+  for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x) {
+    const Run rn = run_info(a, run);
+    if (rn.unit != prev_unit) {
+      prev_unit = rn.unit;
+      u = unit_info(a, rn.unit);
+      if (jl == 0) {
+        *(volatile int*)&sh->p2_unit = rn.unit;            // lets pass 1 move on (see producer)
+        int ready = 1;
         const long long t0 = now_ns();
-        while (ld_acquire(&a.flag[unit]) < 128) {
+        while (ld_acquire(&a.flag[rn.unit]) < 128) {
           __nanosleep(200);
           if (now_ns() - t0 > kWaitLimitNs) {
             atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
-            dead = true;
+            ready = 0;
             break;
           }
         }
+        sh->p2_ready = ready;
       }
-      group_sync(2);                                    // everyone is done with the previous constants
-      if (jl < u.npad) {
-        const int i = obs_row(a, u, jl);
+      group_sync(2);                                       // flag seen; everyone is done with the old constants
+      if (sh->p2_ready == 0) dead = true;
+      {
         const bool live = jl < u.rows && !dead;
-        row_const[jl] = make_float2(live ? c_smem[i] : 0.f,
-                                    live ? __ldcg(&a.final_off[(size_t)unit * 128 + jl]) : INFINITY);
+        const int i = obs_row(a, u, jl);
+        sh->row_const[jl] = make_float2(live ? sh->c[i] : 0.f,
+                                        live ? __ldcg(&a.final_off[(size_t)rn.unit * 128 + jl]) : INFINITY);
       }
       group_sync(2);
     }
-    const int acc = it & 1, aph = (it >> 1) & 1;
-    if (!gone && !mbar_wait(&bars->acc_full[1][acc], aph, a.status)) gone = true;
-    if (gone) continue;  // only the unit-change barriers above remain
-    tc_fence_after();
-    const int j = blk * kKeyTile + jl;
-    const bool full = blk * kKeyTile + kKeyTile - 1 <= a.n - a.r;
-    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((2 + acc) * 128);
-    float sum = 0.f;
-    // npad is a multiple of 16 and the product wrote exactly npad columns: never read beyond them.
-    // Rows between `rows` and npad are zero rows of Q with weight 0 and offset +inf: 2^{-inf} = 0.
-#pragma unroll 1
-    for (int ch = 0; ch * 16 < u.npad; ++ch) {
-      float v[16];
-      tmem_ld16(taddr + ch * 16, v);
+    for (int t = 0; t < rn.cnt; ++t, ++it) {
+      if (gone) continue;
+      const int acc = it & 1, aph = (it >> 1) & 1;
+      if (!mbar_wait(&bars->acc_full[1][acc], aph, a.status)) { gone = true; continue; }
+      tc_fence_after();
+      const int j0 = (rn.blk0 + t) * kKeyTile, j = j0 + jl;
+      const bool full = j0 + kKeyTile - 1 <= a.n - a.r;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((2 + acc) * 128);
+      float sum = 0.f;
+      // The product wrote exactly npad (a multiple of 16) columns; rows between `rows` and npad are zero
+      // rows of Q with weight 0 and offset +inf, contributing 2^{-inf} = 0.
       if (full) {
-#pragma unroll
-        for (int t = 0; t < 16; ++t) {
-          const float2 rc = row_const[ch * 16 + t];
-          sum += fast_exp2(fmaf(v[t], rc.x, -rc.y));
+        uint32_t ra[32], rb[32];
+        tmem_ld32_issue(taddr, ra);
+#pragma unroll 1
+        for (int s0 = 0; s0 < u.npad; s0 += 64) {
+          tmem_ld_wait(ra);
+          if (s0 + 32 < u.npad) tmem_ld32_issue(taddr + s0 + 32, rb);
+          sum += column_chunk(ra, rc2, s0, u.npad - s0);
+          if (s0 + 32 < u.npad) {
+            tmem_ld_wait(rb);
+            if (s0 + 64 < u.npad) tmem_ld32_issue(taddr + s0 + 64, ra);
+            sum += column_chunk(rb, rc2, s0 + 32, u.npad - s0 - 32);
+          }
         }
       } else {
+#pragma unroll 1
+        for (int s0 = 0; s0 < u.npad; s0 += 16) {
+          float v[16];
+          tmem_ld16(taddr + s0, v);
 #pragma unroll
-        for (int t = 0; t < 16; ++t) {
-          const int sr = ch * 16 + t;
-          const float2 rc = row_const[sr];
-          const bool vis = sr < u.rows && j <= a.n - a.r + obs_row(a, u, sr);
-          if (vis) sum += fast_exp2(fmaf(v[t], rc.x, -rc.y));
+          for (int t2 = 0; t2 < 16; ++t2) {
+            const int sr = s0 + t2;
+            const float2 rc = sh->row_const[sr];
+            const bool vis = sr < u.rows && j <= a.n - a.r + obs_row(a, u, sr);
+            if (vis) sum += fast_exp2(fmaf(v[t2], rc.x, -rc.y));
+          }
         }
       }
+      tc_fence_before();
+      mbar_arrive(&bars->acc_empty[1][acc]);
+      if (j < a.n) a.s_raw[(size_t)rn.unit * a.n + j] = sum;
     }
-    tc_fence_before();
-    mbar_arrive(&bars->acc_empty[1][acc]);
-    if (j < a.n) a.s_raw[(size_t)unit * a.n + j] = sum;
   }
+  if (jl == 0) *(volatile int*)&sh->p2_unit = 0x3fffffff;   // nothing left for pass 1 to wait for
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -460,15 +576,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   char* tiles = reinterpret_cast<char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   char* q_smem[2] = {tiles, tiles + kQBytes + kKRingBytes};
   char* k_ring[2] = {tiles + kQBytes, tiles + 2 * kQBytes + kKRingBytes};
-  char* misc = tiles + kSmemTiles;
-  Barriers* bars = reinterpret_cast<Barriers*>(misc);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 256);
-  int* bcast = reinterpret_cast<int*>(misc + 272);
-  float* c_smem = reinterpret_cast<float*>(misc + 512);             // [256]
-  float2* row_const = reinterpret_cast<float2*>(misc + 512 + 1024); // [128]
+  Shared* sh = reinterpret_cast<Shared*>(tiles + kSmemTiles);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int t = threadIdx.x; t < kMaxRows; t += kThreads) c_smem[t] = a.c[t];
+  for (int t = threadIdx.x; t < kMaxRows; t += kThreads) sh->c[t] = a.c[t];
+  for (int t = threadIdx.x; t < 128; t += kThreads) sh->row_const[t] = make_float2(0.f, INFINITY);
   // Q rows a TMA box never covers (row blocks with fewer than 128 rows) must read as zeros, not as
   // whatever the last kernel left: zero both Q buffers once, before any bulk copy is issued.
   for (int p = 0; p < 2; ++p) {
@@ -477,6 +589,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (threadIdx.x == 0) {
+    Barriers* bars = &sh->bars;
     for (int p = 0; p < 2; ++p) {
       mbar_init(&bars->q_full[p], 1);
       for (int s = 0; s < kStages; ++s) {
@@ -487,30 +600,37 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
         mbar_init(&bars->acc_full[p][s], 1);
         mbar_init(&bars->acc_empty[p][s], 128);
       }
+      mbar_init(&bars->pub_full[p], 128);
+      mbar_init(&bars->pub_free[p], 128);
     }
+    sh->p2_unit = 0;
+    sh->p2_ready = 1;
+    sh->bcast = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // all 512 TMEM columns: four 128-column accumulators
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(tmem_slot)) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(&sh->tmem_slot)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t tmem_base = sh->tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) producer(a, &qmap, &kmap, bars, 0, q_smem[0], k_ring[0]);
+    if (lane == 0) producer(a, &qmap, &kmap, sh, 0, q_smem[0], k_ring[0]);
   } else if (warp == 1) {
-    if (lane == 0) mma_issuer(a, bars, 0, q_smem[0], k_ring[0], tmem_base);
+    if (lane == 0) mma_issuer(a, sh, 0, q_smem[0], k_ring[0], tmem_base);
   } else if (warp == 2) {
-    if (lane == 0) producer(a, &qmap, &kmap, bars, 1, q_smem[1], k_ring[1]);
+    if (lane == 0) producer(a, &qmap, &kmap, sh, 1, q_smem[1], k_ring[1]);
   } else if (warp == 3) {
-    if (lane == 0) mma_issuer(a, bars, 1, q_smem[1], k_ring[1], tmem_base);
+    if (lane == 0) mma_issuer(a, sh, 1, q_smem[1], k_ring[1], tmem_base);
   } else if (warp < 8) {
-    row_stats_group(a, bars, tmem_base, c_smem, bcast);
+    row_stats_group(a, sh, tmem_base);
+  } else if (warp < 12) {
+    column_sum_group(a, sh, tmem_base);
   } else {
-    column_sum_group(a, bars, tmem_base, c_smem, row_const);
+    publisher_group(a, sh);
   }
 
   tc_fence_before();
@@ -572,10 +692,15 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float
   TcArgs a;
   a.n = pl.n; a.r = pl.r; a.G = pl.G; a.Hkv = pl.Hkv; a.n_rb = pl.n_rb; a.hb = pl.heads_per_rb;
   a.n_blk = pl.n_blk; a.D = pl.d;
-  a.T = units * pl.n_blk;
-  int ch = a.T / (n_sm * 8);
-  a.CH = ch < 1 ? 1 : (ch > 4 ? 4 : ch);
-  a.n_runs = (a.T + a.CH - 1) / a.CH;
+  const long long tiles = (long long)units * pl.n_blk;
+  const long long ch = tiles / ((long long)n_sm * 8);
+  a.CH = ch < 1 ? 1 : (ch > 4 ? 4 : (int)ch);
+  a.rpu = (pl.n_blk + a.CH - 1) / a.CH;
+  a.n_runs = units * a.rpu;
+  // keep about 32 MiB of keys between the two passes
+  const long long unit_bytes = (long long)pl.n * pl.d * pl.es;
+  const long long lag = (32LL << 20) / (unit_bytes * pl.n_rb > 0 ? unit_bytes : 1) * pl.n_rb;
+  a.lag = lag < 2 * pl.n_rb ? 2 * pl.n_rb : (lag > 4096 ? 4096 : (int)lag);
   a.bf16 = pl.dtype == AHAKV_BF16;
   a.log2G = log2f((float)pl.G);
   for (int i = 0; i < kMaxRows; ++i) a.c[i] = pl.rows.c[i];
