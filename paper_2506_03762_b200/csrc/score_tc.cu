@@ -196,19 +196,22 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t* r) {
                : "memory");
 }
 
-// 16 consecutive FP32 columns of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-  uint32_t r[16];
+// 16 consecutive FP32 columns of this thread's TMEM lane: issue now, use after tmem_ld_wait16(r).
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr)
       : "memory");
-#pragma unroll
-  for (int t = 0; t < 16; ++t) v[t] = __uint_as_float(r[t]);
+}
+__device__ __forceinline__ void tmem_ld_wait16(uint32_t* r) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :
+               : "memory");
 }
 
 __device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
@@ -339,7 +342,13 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, int pipe, char* q_smem, 
   }
 }
 
-// One 32-key chunk of a row: fold (max, sum of 2^{c w - max}) into the running pair.
+// One 32-key chunk of a row: fold it into the running pair (M, Z) with Z = sum of 2^{c w - M}.
+// M is a shift, not necessarily the maximum: any value within 2^kShiftSlack of the largest logit seen
+// keeps every term finite, so the exponentials of a chunk are taken against the shift the row already
+// has, without waiting for the chunk's own maximum; only when that maximum outruns the shift by more
+// than the slack (or the row has no shift yet) is the chunk redone against a new shift.
+constexpr float kShiftSlack = 64.f;
+
 __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_first, int last, float c, float& M,
                                            float& Z) {
   float v[32];
@@ -356,10 +365,9 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
     mx0 = fmaxf(mx0, fmaxf(v[t], v[t + 1]));
     mx1 = fmaxf(mx1, fmaxf(v[t + 2], v[t + 3]));
   }
-  const float mx = fmaxf(mx0, mx1);
-  if (mx > -INFINITY) {
-    const float m2 = fmaxf(mx * c, M);          // the running maximum after this chunk
-    const float neg = -m2;
+  const float mx = fmaxf(mx0, mx1) * c;
+  if (M > -INFINITY) {
+    const float neg = -M;
     float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
 #pragma unroll
     for (int t = 0; t < 32; t += 4) {
@@ -368,9 +376,23 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
       z2 += fast_exp2(fmaf(v[t + 2], c, neg));
       z3 += fast_exp2(fmaf(v[t + 3], c, neg));
     }
-    if (m2 > M) Z *= fast_exp2(M - m2);          // rare once the maximum has settled
-    Z += (z0 + z1) + (z2 + z3);
-    M = m2;
+    if (mx <= M + kShiftSlack) {
+      Z += (z0 + z1) + (z2 + z3);
+      return;
+    }
+  }
+  if (mx > -INFINITY) {                              // first visible keys of the row, or the shift fell behind
+    const float neg = -mx;
+    float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+#pragma unroll
+    for (int t = 0; t < 32; t += 4) {
+      z0 += fast_exp2(fmaf(v[t], c, neg));
+      z1 += fast_exp2(fmaf(v[t + 1], c, neg));
+      z2 += fast_exp2(fmaf(v[t + 2], c, neg));
+      z3 += fast_exp2(fmaf(v[t + 3], c, neg));
+    }
+    Z = (M > -INFINITY ? Z * fast_exp2(M - mx) : 0.f) + ((z0 + z1) + (z2 + z3));
+    M = mx;
   }
 }
 
@@ -470,25 +492,32 @@ __device__ void publisher_group(const TcArgs& a, Shared* sh) {
   }
 }
 
-// One 32-row chunk of a key's column: add 2^{c w - off} over rows [s0, s0 + cols).
-__device__ __forceinline__ float column_chunk(const uint32_t* r, const float4* rc2, int s0, int cols) {
-  float z0 = 0.f, z1 = 0.f;
+// (c, off) of sixteen consecutive stacked rows, as eight 128-bit shared-memory loads.  Volatile, so that
+// the loads stay where they are written: ahead of the arithmetic on the chunk before.
+__device__ __forceinline__ void ld_row_consts(const float2* row_const, int s0, float4* k) {
+  const uint32_t addr = smem_u32(row_const + s0);
 #pragma unroll
-  for (int t = 0; t < 32; t += 2) {
-    if (t < 16 || cols > 16) {
-      const float4 k = rc2[(s0 + t) >> 1];                 // (c, off) of two consecutive rows
-      z0 += fast_exp2(fmaf(__uint_as_float(r[t]), k.x, -k.y));
-      z1 += fast_exp2(fmaf(__uint_as_float(r[t + 1]), k.z, -k.w));
-    }
+  for (int t = 0; t < 8; ++t)
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(k[t].x), "=f"(k[t].y), "=f"(k[t].z), "=f"(k[t].w) : "r"(addr + 16 * t));
+}
+
+// Sixteen stacked rows of a key's column: adds 2^{c w - off} of each into four partial sums.
+__device__ __forceinline__ void column_chunk16(const uint32_t* r, const float4* k, float& z0, float& z1, float& z2,
+                                               float& z3) {
+#pragma unroll
+  for (int t = 0; t < 8; t += 2) {
+    z0 += fast_exp2(fmaf(__uint_as_float(r[2 * t]), k[t].x, -k[t].y));
+    z1 += fast_exp2(fmaf(__uint_as_float(r[2 * t + 1]), k[t].z, -k[t].w));
+    z2 += fast_exp2(fmaf(__uint_as_float(r[2 * t + 2]), k[t + 1].x, -k[t + 1].y));
+    z3 += fast_exp2(fmaf(__uint_as_float(r[2 * t + 3]), k[t + 1].z, -k[t + 1].w));
   }
-  return z0 + z1;
 }
 
 // Pass-2 softmax group: thread `jl` owns key j0 + jl.
 __device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base) {
   Barriers* bars = &sh->bars;
   const int jl = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
-  const float4* rc2 = reinterpret_cast<const float4*>(sh->row_const);
   int it = 0, prev_unit = -1;
   bool dead = false;     // a flag wait ran out: keep the pipeline protocol, skip the arithmetic
   bool gone = false;     // an accumulator wait ran out: keep only the group barriers
@@ -534,30 +563,44 @@ __device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base
       // The product wrote exactly npad (a multiple of 16) columns; rows between `rows` and npad are zero
       // rows of Q with weight 0 and offset +inf, contributing 2^{-inf} = 0.
       if (full) {
-        uint32_t ra[32], rb[32];
-        tmem_ld32_issue(taddr, ra);
+        // Two chunks are in flight at any time: while one is summed, the next one's accumulator columns
+        // and row constants are already on their way.
+        uint32_t ra[16], rb[16];
+        float4 ka[8], kb[8];
+        float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+        tmem_ld16_issue(taddr, ra);
+        ld_row_consts(sh->row_const, 0, ka);
 #pragma unroll 1
-        for (int s0 = 0; s0 < u.npad; s0 += 64) {
-          tmem_ld_wait(ra);
-          if (s0 + 32 < u.npad) tmem_ld32_issue(taddr + s0 + 32, rb);
-          sum += column_chunk(ra, rc2, s0, u.npad - s0);
-          if (s0 + 32 < u.npad) {
-            tmem_ld_wait(rb);
-            if (s0 + 64 < u.npad) tmem_ld32_issue(taddr + s0 + 64, ra);
-            sum += column_chunk(rb, rc2, s0 + 32, u.npad - s0 - 32);
+        for (int s0 = 0; s0 < u.npad; s0 += 32) {
+          const bool more = s0 + 16 < u.npad;
+          tmem_ld_wait16(ra);
+          if (more) {
+            tmem_ld16_issue(taddr + s0 + 16, rb);
+            ld_row_consts(sh->row_const, s0 + 16, kb);
+          }
+          column_chunk16(ra, ka, z0, z1, z2, z3);
+          if (more) {
+            tmem_ld_wait16(rb);
+            if (s0 + 32 < u.npad) {
+              tmem_ld16_issue(taddr + s0 + 32, ra);
+              ld_row_consts(sh->row_const, s0 + 32, ka);
+            }
+            column_chunk16(rb, kb, z0, z1, z2, z3);
           }
         }
+        sum = (z0 + z1) + (z2 + z3);
       } else {
 #pragma unroll 1
         for (int s0 = 0; s0 < u.npad; s0 += 16) {
-          float v[16];
-          tmem_ld16(taddr + s0, v);
+          uint32_t v[16];
+          tmem_ld16_issue(taddr + s0, v);
+          tmem_ld_wait16(v);
 #pragma unroll
           for (int t2 = 0; t2 < 16; ++t2) {
             const int sr = s0 + t2;
             const float2 rc = sh->row_const[sr];
             const bool vis = sr < u.rows && j <= a.n - a.r + obs_row(a, u, sr);
-            if (vis) sum += fast_exp2(fmaf(v[t2], rc.x, -rc.y));
+            if (vis) sum += fast_exp2(fmaf(__uint_as_float(v[t2]), rc.x, -rc.y));
           }
         }
       }
@@ -697,9 +740,9 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float
   a.CH = ch < 1 ? 1 : (ch > 4 ? 4 : (int)ch);
   a.rpu = (pl.n_blk + a.CH - 1) / a.CH;
   a.n_runs = units * a.rpu;
-  // keep about 32 MiB of keys between the two passes
+  // keep about 64 MiB of keys between the two passes: half of L2
   const long long unit_bytes = (long long)pl.n * pl.d * pl.es;
-  const long long lag = (32LL << 20) / (unit_bytes * pl.n_rb > 0 ? unit_bytes : 1) * pl.n_rb;
+  const long long lag = (64LL << 20) / (unit_bytes * pl.n_rb > 0 ? unit_bytes : 1) * pl.n_rb;
   a.lag = lag < 2 * pl.n_rb ? 2 * pl.n_rb : (lag > 4096 ? 4096 : (int)lag);
   a.bf16 = pl.dtype == AHAKV_BF16;
   a.log2G = log2f((float)pl.G);
