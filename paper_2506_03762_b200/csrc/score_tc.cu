@@ -34,7 +34,7 @@ namespace {
 
 constexpr int kStages = 2;                 // K-tile ring depth per pipeline
 constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 16-bit elements, 128-byte swizzled
-constexpr int kThreads = 512;              // 4 service warps + two softmax groups + the publisher group
+constexpr int kThreads = 768;              // 4 service warps, 8 + 8 softmax warps, the 4-warp publisher group
 constexpr long long kWaitLimitNs = 1000000000LL;   // 1 s
 
 struct TcArgs {
@@ -73,7 +73,8 @@ struct Shared {
   int p2_ready;
   float c[kMaxRows];            // lambda_i * log2(e) per observation row
   float2 row_const[128];        // pass 2: (c, offset) per stacked row of the current row block
-  float2 pub[2][128];           // pass 1 -> publisher
+  float2 pub[2][256];           // pass 1 (both column halves) -> publisher
+  float p2_part[2][128];        // pass 2: partial column sums of the second half of the rows
 };
 
 constexpr int kQBytes = 2 * kSubTileBytes;              // per pipeline, D <= 128
@@ -214,7 +215,9 @@ __device__ __forceinline__ void tmem_ld_wait16(uint32_t* r) {
                : "memory");
 }
 
-__device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+__device__ __forceinline__ void group_sync(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
 
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;
@@ -396,9 +399,10 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
   }
 }
 
-// Pass-1 softmax group: thread `s` owns stacked row s.  One (max, sum) pair per run goes to the
-// publisher group through shared memory, so this group never waits on global memory.
-__device__ void row_stats_group(const TcArgs& a, Shared* sh, uint32_t tmem_base) {
+// Pass-1 softmax groups: two groups of four warps share each accumulator; thread `s` of group `half`
+// owns stacked row s over key columns [64 half, 64 half + 64) of the tile.  One (shift, sum) pair per run
+// and half goes to the publisher group through shared memory, so these groups never wait on global memory.
+__device__ void row_stats_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int half) {
   Barriers* bars = &sh->bars;
   const int s = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
   int it = 0, run_it = 0;
@@ -414,29 +418,25 @@ __device__ void row_stats_group(const TcArgs& a, Shared* sh, uint32_t tmem_base)
       const int acc = it & 1, aph = (it >> 1) & 1;
       if (!mbar_wait(&bars->acc_full[0][acc], aph, a.status)) { dead = true; break; }
       tc_fence_after();
-      const int j0 = (rn.blk0 + t) * kKeyTile;
-      const bool full = j0 + kKeyTile - 1 <= a.n - a.r;   // every key of the tile is visible to every row
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 128);
-      uint32_t ra[32], rb[32];
+      const int j0 = (rn.blk0 + t) * kKeyTile + 64 * half;
+      const bool full = (rn.blk0 + t) * kKeyTile + kKeyTile - 1 <= a.n - a.r;   // no key of the tile is masked
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 128 + 64 * half);
+      uint32_t ra[32];
+      // One chunk at a time: load, wait, fold.  The other warps of the scheduler fill the load latency;
+      // keeping a second load in flight costs registers and ties the exponentials to its completion.
       tmem_ld32_issue(taddr, ra);
       tmem_ld_wait(ra);
-      tmem_ld32_issue(taddr + 32, rb);
       fold_chunk(ra, full, j0, last, c, M, Z);
-      tmem_ld_wait(rb);
-      tmem_ld32_issue(taddr + 64, ra);
-      fold_chunk(rb, full, j0 + 32, last, c, M, Z);
+      tmem_ld32_issue(taddr + 32, ra);
       tmem_ld_wait(ra);
-      tmem_ld32_issue(taddr + 96, rb);
-      fold_chunk(ra, full, j0 + 64, last, c, M, Z);
-      tmem_ld_wait(rb);
       tc_fence_before();
       mbar_arrive(&bars->acc_empty[0][acc]);               // the accumulator is free for the next product
-      fold_chunk(rb, full, j0 + 96, last, c, M, Z);
+      fold_chunk(ra, full, j0 + 32, last, c, M, Z);
     }
     if (dead) break;
     const int slot = run_it & 1, sph = (run_it >> 1) & 1;
     if (!mbar_wait(&bars->pub_free[slot], sph ^ 1, a.status)) break;
-    sh->pub[slot][s] = make_float2(M, Z);
+    sh->pub[slot][128 * half + s] = make_float2(M, Z);
     mbar_arrive(&bars->pub_full[slot]);
   }
 }
@@ -453,16 +453,19 @@ __device__ void publisher_group(const TcArgs& a, Shared* sh) {
     const int slot = run_it & 1, sph = (run_it >> 1) & 1;
     if (!dead && !mbar_wait(&bars->pub_full[slot], sph, a.status)) dead = true;
     if (!dead) {
-      const float2 e = sh->pub[slot][s];
+      const float2 e0 = sh->pub[slot][s], e1 = sh->pub[slot][128 + s];   // the two column halves of the row
       mbar_arrive(&bars->pub_free[slot]);
+      float2 e;
+      e.x = fmaxf(e0.x, e1.x);
+      e.y = (e0.y > 0.f ? e0.y * fast_exp2(e0.x - e.x) : 0.f) + (e1.y > 0.f ? e1.y * fast_exp2(e1.x - e.x) : 0.f);
       a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s] = e;
       __threadfence();
     }
-    group_sync(3);
+    group_sync(3, 128);
     if (s == 0) sh->bcast = dead ? -1 : atomicAdd(&a.cnt[rn.unit], 1);
-    group_sync(3);
+    group_sync(3, 128);
     const bool last_run = sh->bcast == a.rpu - 1;
-    group_sync(3);                                         // bcast may be rewritten after this point
+    group_sync(3, 128);                                         // bcast may be rewritten after this point
     if (last_run && !dead) {
       __threadfence();
       const float2* p = a.partial + (size_t)rn.unit * a.rpu * 128 + s;
@@ -514,20 +517,26 @@ __device__ __forceinline__ void column_chunk16(const uint32_t* r, const float4* 
   }
 }
 
-// Pass-2 softmax group: thread `jl` owns key j0 + jl.
-__device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base) {
+// Pass-2 softmax groups: two groups of four warps share each accumulator; thread `jl` of either group owns
+// key j0 + jl, group 0 over the first half of the stacked rows (accumulator columns), group 1 over the
+// rest.  Group 1 hands its partial sum over through shared memory; group 0 adds the two and stores.
+__device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int half) {
   Barriers* bars = &sh->bars;
   const int jl = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
   int it = 0, prev_unit = -1;
   bool dead = false;     // a flag wait ran out: keep the pipeline protocol, skip the arithmetic
   bool gone = false;     // an accumulator wait ran out: keep only the group barriers
   UnitInfo u = unit_info(a, 0);
+  int c_lo = 0, c_hi = 0;   // this group's accumulator columns
   for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x) {
     const Run rn = run_info(a, run);
     if (rn.unit != prev_unit) {
       prev_unit = rn.unit;
       u = unit_info(a, rn.unit);
-      if (jl == 0) {
+      const int split = ((u.npad / 16 + 1) / 2) * 16;
+      c_lo = half ? split : 0;
+      c_hi = half ? u.npad : split;
+      if (half == 0 && jl == 0) {
         *(volatile int*)&sh->p2_unit = rn.unit;            // lets pass 1 move on (see producer)
         int ready = 1;
         const long long t0 = now_ns();
@@ -541,75 +550,65 @@ __device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base
         }
         sh->p2_ready = ready;
       }
-      group_sync(2);                                       // flag seen; everyone is done with the old constants
+      group_sync(2, 256);                                  // flag seen; everyone is done with the old constants
       if (sh->p2_ready == 0) dead = true;
-      {
+      if (half == 0) {
         const bool live = jl < u.rows && !dead;
         const int i = obs_row(a, u, jl);
         sh->row_const[jl] = make_float2(live ? sh->c[i] : 0.f,
                                         live ? __ldcg(&a.final_off[(size_t)rn.unit * 128 + jl]) : INFINITY);
       }
-      group_sync(2);
+      group_sync(2, 256);
     }
     for (int t = 0; t < rn.cnt; ++t, ++it) {
-      if (gone) continue;
       const int acc = it & 1, aph = (it >> 1) & 1;
-      if (!mbar_wait(&bars->acc_full[1][acc], aph, a.status)) { gone = true; continue; }
-      tc_fence_after();
       const int j0 = (rn.blk0 + t) * kKeyTile, j = j0 + jl;
-      const bool full = j0 + kKeyTile - 1 <= a.n - a.r;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((2 + acc) * 128);
       float sum = 0.f;
-      // The product wrote exactly npad (a multiple of 16) columns; rows between `rows` and npad are zero
-      // rows of Q with weight 0 and offset +inf, contributing 2^{-inf} = 0.
-      if (full) {
-        // Two chunks are in flight at any time: while one is summed, the next one's accumulator columns
-        // and row constants are already on their way.
-        uint32_t ra[16], rb[16];
-        float4 ka[8], kb[8];
-        float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
-        tmem_ld16_issue(taddr, ra);
-        ld_row_consts(sh->row_const, 0, ka);
+      if (!gone && !mbar_wait(&bars->acc_full[1][acc], aph, a.status)) gone = true;
+      if (!gone) {
+        tc_fence_after();
+        const bool full = j0 + kKeyTile - 1 <= a.n - a.r;
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((2 + acc) * 128);
+        // The product wrote exactly npad (a multiple of 16) columns; rows between `rows` and npad are zero
+        // rows of Q with weight 0 and offset +inf, contributing 2^{-inf} = 0.
+        if (full) {
+          uint32_t ra[16];
+          float4 ka[8];
+          float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
 #pragma unroll 1
-        for (int s0 = 0; s0 < u.npad; s0 += 32) {
-          const bool more = s0 + 16 < u.npad;
-          tmem_ld_wait16(ra);
-          if (more) {
-            tmem_ld16_issue(taddr + s0 + 16, rb);
-            ld_row_consts(sh->row_const, s0 + 16, kb);
+          for (int s0 = c_lo; s0 < c_hi; s0 += 16) {
+            tmem_ld16_issue(taddr + s0, ra);
+            ld_row_consts(sh->row_const, s0, ka);
+            tmem_ld_wait16(ra);
+            column_chunk16(ra, ka, z0, z1, z2, z3);
           }
-          column_chunk16(ra, ka, z0, z1, z2, z3);
-          if (more) {
-            tmem_ld_wait16(rb);
-            if (s0 + 32 < u.npad) {
-              tmem_ld16_issue(taddr + s0 + 32, ra);
-              ld_row_consts(sh->row_const, s0 + 32, ka);
-            }
-            column_chunk16(rb, kb, z0, z1, z2, z3);
-          }
-        }
-        sum = (z0 + z1) + (z2 + z3);
-      } else {
+          sum = (z0 + z1) + (z2 + z3);
+        } else {
 #pragma unroll 1
-        for (int s0 = 0; s0 < u.npad; s0 += 16) {
-          uint32_t v[16];
-          tmem_ld16_issue(taddr + s0, v);
-          tmem_ld_wait16(v);
+          for (int s0 = c_lo; s0 < c_hi; s0 += 16) {
+            uint32_t v[16];
+            tmem_ld16_issue(taddr + s0, v);
+            tmem_ld_wait16(v);
 #pragma unroll
-          for (int t2 = 0; t2 < 16; ++t2) {
-            const int sr = s0 + t2;
-            const float2 rc = sh->row_const[sr];
-            const bool vis = sr < u.rows && j <= a.n - a.r + obs_row(a, u, sr);
-            if (vis) sum += fast_exp2(fmaf(__uint_as_float(v[t2]), rc.x, -rc.y));
+            for (int t2 = 0; t2 < 16; ++t2) {
+              const int sr = s0 + t2;
+              const float2 rc = sh->row_const[sr];
+              const bool vis = sr < u.rows && j <= a.n - a.r + obs_row(a, u, sr);
+              if (vis) sum += fast_exp2(fmaf(__uint_as_float(v[t2]), rc.x, -rc.y));
+            }
           }
         }
+        tc_fence_before();
+        mbar_arrive(&bars->acc_empty[1][acc]);
       }
-      tc_fence_before();
-      mbar_arrive(&bars->acc_empty[1][acc]);
-      if (j < a.n) a.s_raw[(size_t)rn.unit * a.n + j] = sum;
+      // Both groups meet here once per tile, also after a wait has run out, so that nobody is left at
+      // the barrier.  Two slots: group 1 can be at most one tile ahead of group 0's read.
+      if (half == 1) sh->p2_part[it & 1][jl] = sum;
+      group_sync(4, 256);
+      if (half == 0 && !gone && j < a.n) a.s_raw[(size_t)rn.unit * a.n + j] = sum + sh->p2_part[it & 1][jl];
     }
   }
-  if (jl == 0) *(volatile int*)&sh->p2_unit = 0x3fffffff;   // nothing left for pass 1 to wait for
+  if (half == 0 && jl == 0) *(volatile int*)&sh->p2_unit = 0x3fffffff;   // nothing left for pass 1 to wait for
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -641,9 +640,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
       }
       for (int s = 0; s < 2; ++s) {
         mbar_init(&bars->acc_full[p][s], 1);
-        mbar_init(&bars->acc_empty[p][s], 128);
+        mbar_init(&bars->acc_empty[p][s], 256);
       }
-      mbar_init(&bars->pub_full[p], 128);
+      mbar_init(&bars->pub_full[p], 256);
       mbar_init(&bars->pub_free[p], 128);
     }
     sh->p2_unit = 0;
@@ -668,10 +667,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     if (lane == 0) producer(a, &qmap, &kmap, sh, 1, q_smem[1], k_ring[1]);
   } else if (warp == 3) {
     if (lane == 0) mma_issuer(a, sh, 1, q_smem[1], k_ring[1], tmem_base);
-  } else if (warp < 8) {
-    row_stats_group(a, sh, tmem_base);
   } else if (warp < 12) {
-    column_sum_group(a, sh, tmem_base);
+    row_stats_group(a, sh, tmem_base, (warp - 4) >> 2);
+  } else if (warp < 20) {
+    column_sum_group(a, sh, tmem_base, (warp - 12) >> 2);
   } else {
     publisher_group(a, sh);
   }
