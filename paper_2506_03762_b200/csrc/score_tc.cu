@@ -11,16 +11,23 @@
 //                                 of the tile, written as a partial; the CTA that
 //                                 delivers a row block's last partial merges them
 //                                 into one offset per row and raises the block's flag.
-//   pass 2 (keys on TMEM lanes):  D = K . Q^T   -> each thread owns one key and adds
-//                                 2^{c w - offset} over the rows: the column sum
-//                                 needs no cross-thread traffic at all.
+//   pass 2 (keys on TMEM lanes):  D = K . Q^T - off/c -> each thread owns one key and adds
+//                                 2^{c D} over the rows: the column sum needs no
+//                                 cross-thread traffic and no per-row constant but c.
 //
 // Both products are tcgen05.mma kind::f16 with FP32 accumulators in TMEM, fed by
 // TMA (128-byte swizzle) from the same K-major Q and K tiles, which serve as A or
 // B operand alike.  Pass 2 trails pass 1 by a few row blocks, so its second read
 // of K is served by L2 and HBM sees K once.
 //
-// Each pipeline has its own TMA warp, MMA warp and 4-warp softmax group; pass 1
+// The row offsets of pass 2 ride in the product itself: the CTA that finishes a row
+// block's statistics writes, per row, -off/(c kFold) as a sum of three 16-bit numbers
+// into a 16-element extension of the row, and pass 2 appends one more k-step of the
+// MMA that multiplies this extension with a constant tile holding kFold.  The three
+// parts carry 24 (bfloat16) or 33 (float16) significant bits, the products are exact
+// and the accumulator is FP32, so D = w - off/c to FP32 rounding.
+//
+// Each pipeline has its own TMA warp, MMA warp and two 4-warp softmax groups; pass 1
 // never waits on pass 2, so the flag waits of pass 2 cannot deadlock.  The kernel
 // is launched cooperatively with at most one CTA per SM, which guarantees that
 // the CTAs a flag depends on are running.  Every wait is bounded in time; on
@@ -36,6 +43,7 @@ constexpr int kStages = 2;                 // K-tile ring depth per pipeline
 constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 16-bit elements, 128-byte swizzled
 constexpr int kThreads = 768;              // 4 service warps, 8 + 8 softmax warps, the 4-warp publisher group
 constexpr long long kWaitLimitNs = 1000000000LL;   // 1 s
+constexpr float kFold = 256.f;             // value of the constant tile; offsets are stored divided by it
 
 struct TcArgs {
   int n, r, G, Hkv, n_rb, hb, n_blk, D;
@@ -45,9 +53,10 @@ struct TcArgs {
   int lag;        // pass 1 may lead this CTA's pass 2 by at most this many row blocks
   int bf16;       // operand type of the products
   float log2G;
-  float c[kMaxRows];
+  float c[kMaxRows];     // lambda_i log2(e) per observation row
+  float cs[128];         // the same per stacked row of a row block (r <= 128 only)
   float2* partial;   // [unit][run][128]
-  float* final_off;  // [unit][128]
+  uint16_t* qx;      // [unit][128][16] 16-bit: the rows' offset extensions
   float* s_raw;      // [unit][n]
   int* cnt;          // [unit] partials delivered
   int* flag;         // [unit] rows whose offset is ready (128 = all)
@@ -70,16 +79,16 @@ struct Shared {
   uint32_t tmem_slot;
   int bcast;
   int p2_unit;                  // row block pass 2 of this CTA is working on
-  int p2_ready;
   float c[kMaxRows];            // lambda_i * log2(e) per observation row
-  float2 row_const[128];        // pass 2: (c, offset) per stacked row of the current row block
+  float cs2[2][128];            // c per stacked row, by row block parity (r > 128 has two kinds of block)
   float2 pub[2][256];           // pass 1 (both column halves) -> publisher
   float p2_part[2][128];        // pass 2: partial column sums of the second half of the rows
 };
 
 constexpr int kQBytes = 2 * kSubTileBytes;              // per pipeline, D <= 128
 constexpr int kKRingBytes = kStages * 2 * kSubTileBytes;
-constexpr int kSmemTiles = 2 * (kQBytes + kKRingBytes);  // 192 KiB
+constexpr int kExtBytes = 128 * 32;                      // 128 rows x 16 16-bit elements, 32-byte swizzled
+constexpr int kSmemTiles = 2 * (kQBytes + kKRingBytes) + 2 * kExtBytes;  // 200 KiB
 constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 8192 /*barriers, constants*/;
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
@@ -132,6 +141,13 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, v
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -149,6 +165,18 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
   d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset
   d |= (uint64_t)1 << 46;                               // version
   d |= (uint64_t)2 << 61;                               // SWIZZLE_128B
+  return d;
+}
+
+// The same for a K-major tile of 32-byte rows (16 elements, one k-step), 32-byte swizzle, 8-row groups
+// 256 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc_ext(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3ffff) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(256 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)6 << 61;                               // SWIZZLE_32B
   return d;
 }
 
@@ -262,8 +290,8 @@ __device__ __forceinline__ int obs_row(const TcArgs& a, const UnitInfo& u, int s
 // ---- roles --------------------------------------------------------------------------------------------
 // TMA producer of one pipeline.  The pass-1 producer also keeps pass 1 from running more than `lag` row
 // blocks ahead of this CTA's pass 2, so that the keys pass 2 re-reads are still in L2.
-__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, Shared* sh, int pipe,
-                         char* q_smem, char* k_ring) {
+__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, const CUtensorMap* xmap,
+                         Shared* sh, int pipe, char* q_smem, char* k_ring, char* ext_smem) {
   Barriers* bars = &sh->bars;
   const int n_sub = a.D / 64;
   const int q_rows = a.r <= 128 ? a.hb * a.r : 128;
@@ -286,10 +314,27 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
       if (!ok) break;
     }
     if (rn.unit != prev_unit) {
+      if (pipe == 1) {
+        // Pass 2 may start on a row block once its statistics are complete: the offset extension of
+        // its rows is then in global memory.
+        *(volatile int*)&sh->p2_unit = rn.unit;              // lets pass 1 move on (see above)
+        const long long t0 = now_ns();
+        while (ld_acquire(&a.flag[rn.unit]) < 128) {
+          __nanosleep(100);
+          if (now_ns() - t0 > kWaitLimitNs) {
+            atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
+            ok = false;
+            break;
+          }
+        }
+        if (!ok) break;
+        asm volatile("fence.proxy.async;" ::: "memory");     // the extension was written with plain stores
+      }
       // the Q buffer is free once every product issued so far has completed
       if (it > 0) ok = mbar_wait(&bars->k_empty[pipe][(it - 1) % kStages], ((it - 1) / kStages) & 1, a.status);
       if (!ok) break;
-      mbar_expect_tx(&bars->q_full[pipe], q_bytes);
+      mbar_expect_tx(&bars->q_full[pipe], q_bytes + (pipe == 1 ? kExtBytes : 0));
+      if (pipe == 1) tma_load_3d(ext_smem, xmap, &bars->q_full[pipe], 0, 0, rn.unit);
       for (int s = 0; s < n_sub; ++s) {
         if (a.r <= 128) tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[pipe], s * 64, 0, u.h * a.G + u.rb * a.hb, u.b);
         else tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[pipe], s * 64, u.rb * 128, u.h, u.b);
@@ -306,6 +351,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
                     (rn.blk0 + t) * kKeyTile, u.h, u.b);
     }
   }
+  if (pipe == 1) *(volatile int*)&sh->p2_unit = 0x3fffffff;   // nothing left for pass 1 to wait for
   if (!ok) {
     // wind down: give copies already in flight a bounded time (1 ms) to land before the CTA exits
     const long long t0 = now_ns();
@@ -314,7 +360,8 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
 }
 
 // MMA issuer of one pipeline.  pipe 0: D[rows x keys] = Q K^T.  pipe 1: D[keys x rows] = K Q^T.
-__device__ void mma_issuer(const TcArgs& a, Shared* sh, int pipe, char* q_smem, char* k_ring, uint32_t tmem_base) {
+__device__ void mma_issuer(const TcArgs& a, Shared* sh, int pipe, char* q_smem, char* k_ring, char* ext_smem,
+                           char* fold_smem, uint32_t tmem_base) {
   Barriers* bars = &sh->bars;
   int it = 0, prev_unit = -1, q_loads = 0;
   uint32_t idesc = umma_idesc(128, 128, a.bf16);
@@ -339,6 +386,8 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, int pipe, char* q_smem, 
         if (pipe == 0) umma(d_tmem, qd, kd, idesc, kk > 0);
         else umma(d_tmem, kd, qd, idesc, kk > 0);
       }
+      // pass 2: D -= off / c, as one more k-step over the constant tile and the rows' offset extensions
+      if (pipe == 1) umma(d_tmem, umma_desc_ext(smem_u32(fold_smem)), umma_desc_ext(smem_u32(ext_smem)), idesc, 1);
       tc_commit(&bars->k_empty[pipe][stage]);
       tc_commit(&bars->acc_full[pipe][acc]);
     }
@@ -487,47 +536,75 @@ __device__ void publisher_group(const TcArgs& a, Shared* sh) {
           Mx = m;
         }
       }
-      // 2^{c w - off} = softmax weight / G
-      a.final_off[(size_t)rn.unit * 128 + s] = Mx + log2f(Zs) + a.log2G;
+      // 2^{c w - off} = softmax weight / G.  Pass 2 gets -off / (c kFold) as three 16-bit parts, the
+      // first three of the row's sixteen extension elements; the other thirteen are zero.
+      const UnitInfo u = unit_info(a, rn.unit);
+      uint32_t w0 = 0, w1 = 0;
+      if (s < u.rows) {
+        const float off = Mx + log2f(Zs) + a.log2G;
+        float v = -(off / sh->c[obs_row(a, u, s)]) / kFold;
+        if (a.bf16) {
+          const __nv_bfloat16 h1 = __float2bfloat16_rn(v);
+          v -= __bfloat162float(h1);
+          const __nv_bfloat16 h2 = __float2bfloat16_rn(v);
+          v -= __bfloat162float(h2);
+          const __nv_bfloat16 h3 = __float2bfloat16_rn(v);
+          w0 = (uint32_t)__bfloat16_as_ushort(h1) | ((uint32_t)__bfloat16_as_ushort(h2) << 16);
+          w1 = (uint32_t)__bfloat16_as_ushort(h3);
+        } else {
+          v = fminf(fmaxf(v, -60000.f), 60000.f);            // float16 has no room beyond; such logits are not scored
+          const __half h1 = __float2half_rn(v);
+          v -= __half2float(h1);
+          const __half h2 = __float2half_rn(v);
+          v -= __half2float(h2);
+          const __half h3 = __float2half_rn(v);
+          w0 = (uint32_t)__half_as_ushort(h1) | ((uint32_t)__half_as_ushort(h2) << 16);
+          w1 = (uint32_t)__half_as_ushort(h3);
+        }
+      }
+      uint4* row = reinterpret_cast<uint4*>(a.qx + ((size_t)rn.unit * 128 + s) * 16);
+      row[0] = make_uint4(w0, w1, 0u, 0u);
+      row[1] = make_uint4(0u, 0u, 0u, 0u);
       __threadfence();
+      asm volatile("fence.proxy.async;" ::: "memory");     // the rows are read back by bulk tensor copies
       atomicAdd(&a.flag[rn.unit], 1);                      // the block is ready when all 128 rows have reported
     }
   }
 }
 
-// (c, off) of sixteen consecutive stacked rows, as eight 128-bit shared-memory loads.  Volatile, so that
-// the loads stay where they are written: ahead of the arithmetic on the chunk before.
-__device__ __forceinline__ void ld_row_consts(const float2* row_const, int s0, float4* k) {
-  const uint32_t addr = smem_u32(row_const + s0);
+// Sixty-four stacked rows of a key's column, rows [64 HALF, 64 HALF + 64): adds 2^{c D} of each.  The
+// column indices are compile-time constants, so every c comes straight from the kernel's parameter
+// bank as an operand of the multiply.
+template <int HALF>
+__device__ __forceinline__ float column_sum_fast(const TcArgs& a, uint32_t taddr) {
+  float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
 #pragma unroll
-  for (int t = 0; t < 8; ++t)
-    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(k[t].x), "=f"(k[t].y), "=f"(k[t].z), "=f"(k[t].w) : "r"(addr + 16 * t));
-}
-
-// Sixteen stacked rows of a key's column: adds 2^{c w - off} of each into four partial sums.
-__device__ __forceinline__ void column_chunk16(const uint32_t* r, const float4* k, float& z0, float& z1, float& z2,
-                                               float& z3) {
+  for (int q = 0; q < 4; ++q) {
+    uint32_t r[16];
+    tmem_ld16_issue(taddr + 64 * HALF + 16 * q, r);
+    tmem_ld_wait16(r);
 #pragma unroll
-  for (int t = 0; t < 8; t += 2) {
-    z0 += fast_exp2(fmaf(__uint_as_float(r[2 * t]), k[t].x, -k[t].y));
-    z1 += fast_exp2(fmaf(__uint_as_float(r[2 * t + 1]), k[t].z, -k[t].w));
-    z2 += fast_exp2(fmaf(__uint_as_float(r[2 * t + 2]), k[t + 1].x, -k[t + 1].y));
-    z3 += fast_exp2(fmaf(__uint_as_float(r[2 * t + 3]), k[t + 1].z, -k[t + 1].w));
+    for (int t = 0; t < 16; t += 4) {
+      z0 += fast_exp2(__uint_as_float(r[t]) * a.cs[64 * HALF + 16 * q + t]);
+      z1 += fast_exp2(__uint_as_float(r[t + 1]) * a.cs[64 * HALF + 16 * q + t + 1]);
+      z2 += fast_exp2(__uint_as_float(r[t + 2]) * a.cs[64 * HALF + 16 * q + t + 2]);
+      z3 += fast_exp2(__uint_as_float(r[t + 3]) * a.cs[64 * HALF + 16 * q + t + 3]);
+    }
   }
+  return (z0 + z1) + (z2 + z3);
 }
 
 // Pass-2 softmax groups: two groups of four warps share each accumulator; thread `jl` of either group owns
 // key j0 + jl, group 0 over the first half of the stacked rows (accumulator columns), group 1 over the
 // rest.  Group 1 hands its partial sum over through shared memory; group 0 adds the two and stores.
-__device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int half) {
+__device__ __forceinline__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int half) {
   Barriers* bars = &sh->bars;
   const int jl = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
   int it = 0, prev_unit = -1;
-  bool dead = false;     // a flag wait ran out: keep the pipeline protocol, skip the arithmetic
-  bool gone = false;     // an accumulator wait ran out: keep only the group barriers
+  bool gone = false;     // an accumulator wait ran out: keep only the group barrier
   UnitInfo u = unit_info(a, 0);
   int c_lo = 0, c_hi = 0;   // this group's accumulator columns
+  bool fast = false;
   for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x) {
     const Run rn = run_info(a, run);
     if (rn.unit != prev_unit) {
@@ -536,30 +613,9 @@ __device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base
       const int split = ((u.npad / 16 + 1) / 2) * 16;
       c_lo = half ? split : 0;
       c_hi = half ? u.npad : split;
-      if (half == 0 && jl == 0) {
-        *(volatile int*)&sh->p2_unit = rn.unit;            // lets pass 1 move on (see producer)
-        int ready = 1;
-        const long long t0 = now_ns();
-        while (ld_acquire(&a.flag[rn.unit]) < 128) {
-          __nanosleep(200);
-          if (now_ns() - t0 > kWaitLimitNs) {
-            atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
-            ready = 0;
-            break;
-          }
-        }
-        sh->p2_ready = ready;
-      }
-      group_sync(2, 256);                                  // flag seen; everyone is done with the old constants
-      if (sh->p2_ready == 0) dead = true;
-      if (half == 0) {
-        const bool live = jl < u.rows && !dead;
-        const int i = obs_row(a, u, jl);
-        sh->row_const[jl] = make_float2(live ? sh->c[i] : 0.f,
-                                        live ? __ldcg(&a.final_off[(size_t)rn.unit * 128 + jl]) : INFINITY);
-      }
-      group_sync(2, 256);
+      fast = a.r <= 128 && u.rows == 128;
     }
+    const float* cs = sh->cs2[u.rb & 1];
     for (int t = 0; t < rn.cnt; ++t, ++it) {
       const int acc = it & 1, aph = (it >> 1) & 1;
       const int j0 = (rn.blk0 + t) * kKeyTile, j = j0 + jl;
@@ -569,21 +625,10 @@ __device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base
         tc_fence_after();
         const bool full = j0 + kKeyTile - 1 <= a.n - a.r;
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((2 + acc) * 128);
-        // The product wrote exactly npad (a multiple of 16) columns; rows between `rows` and npad are zero
-        // rows of Q with weight 0 and offset +inf, contributing 2^{-inf} = 0.
-        if (full) {
-          uint32_t ra[16];
-          float4 ka[8];
-          float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
-#pragma unroll 1
-          for (int s0 = c_lo; s0 < c_hi; s0 += 16) {
-            tmem_ld16_issue(taddr + s0, ra);
-            ld_row_consts(sh->row_const, s0, ka);
-            tmem_ld_wait16(ra);
-            column_chunk16(ra, ka, z0, z1, z2, z3);
-          }
-          sum = (z0 + z1) + (z2 + z3);
+        if (full && fast) {
+          sum = half ? column_sum_fast<1>(a, taddr) : column_sum_fast<0>(a, taddr);
         } else {
+          // The product wrote exactly npad (a multiple of 16) columns; those past `rows` belong to no row.
 #pragma unroll 1
           for (int s0 = c_lo; s0 < c_hi; s0 += 16) {
             uint32_t v[16];
@@ -592,9 +637,8 @@ __device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base
 #pragma unroll
             for (int t2 = 0; t2 < 16; ++t2) {
               const int sr = s0 + t2;
-              const float2 rc = sh->row_const[sr];
-              const bool vis = sr < u.rows && j <= a.n - a.r + obs_row(a, u, sr);
-              if (vis) sum += fast_exp2(fmaf(__uint_as_float(v[t2]), rc.x, -rc.y));
+              const bool vis = sr < u.rows && (full || j <= a.n - a.r + obs_row(a, u, sr));
+              if (vis) sum += fast_exp2(__uint_as_float(v[t2]) * cs[sr]);
             }
           }
         }
@@ -608,21 +652,33 @@ __device__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base
       if (half == 0 && !gone && j < a.n) a.s_raw[(size_t)rn.unit * a.n + j] = sum + sh->p2_part[it & 1][jl];
     }
   }
-  if (half == 0 && jl == 0) *(volatile int*)&sh->p2_unit = 0x3fffffff;   // nothing left for pass 1 to wait for
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
-                const __grid_constant__ TcArgs a) {
+                const __grid_constant__ CUtensorMap xmap, const __grid_constant__ TcArgs a) {
   extern __shared__ char smem_raw[];
   char* tiles = reinterpret_cast<char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   char* q_smem[2] = {tiles, tiles + kQBytes + kKRingBytes};
   char* k_ring[2] = {tiles + kQBytes, tiles + 2 * kQBytes + kKRingBytes};
+  char* ext_smem = tiles + 2 * (kQBytes + kKRingBytes);   // pass 2: offset extension of the current rows
+  char* fold_smem = ext_smem + kExtBytes;                 // pass 2: the constant tile
   Shared* sh = reinterpret_cast<Shared*>(tiles + kSmemTiles);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int t = threadIdx.x; t < kMaxRows; t += kThreads) sh->c[t] = a.c[t];
-  for (int t = threadIdx.x; t < 128; t += kThreads) sh->row_const[t] = make_float2(0.f, INFINITY);
+  for (int t = threadIdx.x; t < 128; t += kThreads) {
+    sh->cs2[0][t] = a.r <= 128 ? a.c[t % a.r] : a.c[t];
+    sh->cs2[1][t] = a.r <= 128 ? a.c[t % a.r] : a.c[128 + t];
+  }
+  {
+    // every 16-byte chunk of the constant tile reads (kFold, kFold, kFold, 0, 0, 0, 0, 0), whatever
+    // the swizzle does to the order of the chunks; it meets the three parts of the rows' extensions
+    const uint32_t one = a.bf16 ? (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(kFold))
+                                : (uint32_t)__half_as_ushort(__float2half_rn(kFold));
+    uint4* f = reinterpret_cast<uint4*>(fold_smem);
+    for (int t = threadIdx.x; t < kExtBytes / 16; t += kThreads) f[t] = make_uint4(one | (one << 16), one, 0u, 0u);
+  }
   // Q rows a TMA box never covers (row blocks with fewer than 128 rows) must read as zeros, not as
   // whatever the last kernel left: zero both Q buffers once, before any bulk copy is issued.
   for (int p = 0; p < 2; ++p) {
@@ -646,7 +702,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
       mbar_init(&bars->pub_free[p], 128);
     }
     sh->p2_unit = 0;
-    sh->p2_ready = 1;
     sh->bcast = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -660,13 +715,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   const uint32_t tmem_base = sh->tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) producer(a, &qmap, &kmap, sh, 0, q_smem[0], k_ring[0]);
+    if (lane == 0) producer(a, &qmap, &kmap, &xmap, sh, 0, q_smem[0], k_ring[0], ext_smem);
   } else if (warp == 1) {
-    if (lane == 0) mma_issuer(a, sh, 0, q_smem[0], k_ring[0], tmem_base);
+    if (lane == 0) mma_issuer(a, sh, 0, q_smem[0], k_ring[0], ext_smem, fold_smem, tmem_base);
   } else if (warp == 2) {
-    if (lane == 0) producer(a, &qmap, &kmap, sh, 1, q_smem[1], k_ring[1]);
+    if (lane == 0) producer(a, &qmap, &kmap, &xmap, sh, 1, q_smem[1], k_ring[1], ext_smem);
   } else if (warp == 3) {
-    if (lane == 0) mma_issuer(a, sh, 1, q_smem[1], k_ring[1], tmem_base);
+    if (lane == 0) mma_issuer(a, sh, 1, q_smem[1], k_ring[1], ext_smem, fold_smem, tmem_base);
   } else if (warp < 12) {
     row_stats_group(a, sh, tmem_base, (warp - 4) >> 2);
   } else if (warp < 20) {
@@ -714,12 +769,24 @@ bool make_map(CUtensorMap* m, const void* base, int bf16, int d, long long token
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 3-D map {16, 128, units} over the rows' offset extensions, one {16, 128, 1} box per row block, 32-byte swizzle.
+bool make_ext_map(CUtensorMap* m, const void* base, int bf16, long long units) {
+  const cuuint64_t dims[3] = {16, 128, (cuuint64_t)units};
+  const cuuint64_t strides[2] = {32, 128 * 32};
+  const cuuint32_t box[3] = {16, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return encode_fn()(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
+                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                     CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool score_tc_available() { return encode_fn() != nullptr; }
 
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float* s_raw, float2* partial,
-                             float* final_off, int* sync_words, int* status, cudaStream_t st) {
+                             void* row_ext, int* sync_words, int* status, cudaStream_t st) {
   static int n_sm = 0;
   static bool configured = false;
   if (!configured) {
@@ -746,17 +813,19 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float
   a.bf16 = pl.dtype == AHAKV_BF16;
   a.log2G = log2f((float)pl.G);
   for (int i = 0; i < kMaxRows; ++i) a.c[i] = pl.rows.c[i];
-  a.partial = partial; a.final_off = final_off; a.s_raw = s_raw;
+  for (int t = 0; t < 128; ++t) a.cs[t] = pl.r <= 128 ? pl.rows.c[t % pl.r] : 0.f;
+  a.partial = partial; a.qx = static_cast<uint16_t*>(row_ext); a.s_raw = s_raw;
   a.cnt = sync_words; a.flag = sync_words + units; a.status = status;
 
-  CUtensorMap qmap, kmap;
+  CUtensorMap qmap, kmap, xmap;
   const int q_box_rows = pl.r <= 128 ? pl.r : 128, q_box_heads = pl.r <= 128 ? pl.heads_per_rb : 1;
   if (!make_map(&qmap, q, a.bf16, pl.d, pl.r, pl.Hq, pl.B, pl.qs, pl.es, q_box_rows, q_box_heads) ||
-      !make_map(&kmap, k, a.bf16, pl.d, pl.n, pl.Hkv, pl.B, pl.ks, pl.es, kKeyTile, 1))
+      !make_map(&kmap, k, a.bf16, pl.d, pl.n, pl.Hkv, pl.B, pl.ks, pl.es, kKeyTile, 1) ||
+      !make_ext_map(&xmap, row_ext, a.bf16, units))
     return AHAKV_ERR_CUDA;
 
   const int grid = a.n_runs < n_sm ? a.n_runs : n_sm;
-  void* args[] = {&qmap, &kmap, &a};
+  void* args[] = {&qmap, &kmap, &xmap, &a};
   const cudaError_t e = cudaLaunchCooperativeKernel((const void*)score_tc_kernel, dim3(grid), dim3(kThreads), args,
                                                     (size_t)kSmemBytes, st);
   count_launch();
