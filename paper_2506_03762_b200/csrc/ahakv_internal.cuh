@@ -32,7 +32,7 @@ struct Plan {
   long long qs[3], ks[3], vs[3];  // element strides: batch, head, token
   RowScale rows;
   // workspace layout, byte offsets
-  size_t off_status, off_sync, off_sraw, off_nu, off_partial, off_final, off_ext, off_score, ws_total;
+  size_t off_status, off_sync, off_sraw, off_nu, off_partial, off_final, off_score, ws_total;
 };
 
 // plan.cu
@@ -43,7 +43,7 @@ void count_launch(int n = 1);
 ahakv_status launch_score_simt(const Plan& pl, const void* q, const void* k, float* s_raw, float2* partial,
                                float* final_off, cudaStream_t st);
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float* s_raw, float2* partial,
-                             void* row_ext, int* sync_words, int* status, cudaStream_t st);
+                             int* status, cudaStream_t st);
 bool score_tc_available();
 ahakv_status launch_vnorm(const Plan& pl, const void* v, float* nu, cudaStream_t st);
 ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,

@@ -107,7 +107,6 @@ ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
   o.off_nu = off;      off += align_up(units * o.n * sizeof(float), 256);
   o.off_partial = off; off += align_up(units * rb_slots * o.n_blk * (o.use_tc ? 128 : o.R) * sizeof(float2), 256);
   o.off_final = off;   off += align_up(units * rb_slots * (o.use_tc ? 128 : o.R) * sizeof(float2), 256);
-  o.off_ext = off;     off += o.use_tc ? align_up(units * rb_slots * 128 * 16 * 2, 1024) : 0;   // 16-bit row extensions
   o.off_score = off;   off += align_up(units * o.n * sizeof(float), 256);
   o.ws_total = off;
   return AHAKV_OK;
@@ -132,8 +131,7 @@ static ahakv_status queue_score(const Plan& pl, const void* q, const void* k, co
   float2* partial = at<float2>(ws, pl.off_partial);
   float* final_off = at<float>(ws, pl.off_final);
   if (pl.use_tc)
-    rc = launch_score_tc(pl, q, k, s_raw, partial, at<char>(ws, pl.off_ext), at<int>(ws, pl.off_sync),
-                         at<int>(ws, pl.off_status), st);
+    rc = launch_score_tc(pl, q, k, s_raw, partial, at<int>(ws, pl.off_status), st);
   else
     rc = launch_score_simt(pl, q, k, s_raw, partial, final_off, st);
   if (rc) return rc;

@@ -7,10 +7,9 @@
 // first, so every tile is visited twice, by two pipelines that live side by side
 // in each CTA and share nothing but the SM:
 //
-//   pass 1 (rows on TMEM lanes):  D = Q . K^T   -> per-row (max, sum of 2^{c w - max})
-//                                 of the tile, written as a partial; the CTA that
-//                                 delivers a row block's last partial merges them
-//                                 into one offset per row and raises the block's flag.
+//   pass 1 (rows on TMEM lanes):  D = Q . K^T   -> per-row (shift, sum of 2^{c w - shift})
+//                                 of a run of tiles, stored to global memory as one
+//                                 8-byte partial per row and run.
 //   pass 2 (keys on TMEM lanes):  D = K . Q^T - off/c -> each thread owns one key and adds
 //                                 2^{c D} over the rows: the column sum needs no
 //                                 cross-thread traffic and no per-row constant but c.
@@ -20,17 +19,27 @@
 // B operand alike.  Pass 2 trails pass 1 by a few row blocks, so its second read
 // of K is served by L2 and HBM sees K once.
 //
-// The row offsets of pass 2 ride in the product itself: the CTA that finishes a row
-// block's statistics writes, per row, -off/(c kFold) as a sum of three 16-bit numbers
-// into a 16-element extension of the row, and pass 2 appends one more k-step of the
-// MMA that multiplies this extension with a constant tile holding kFold.  The three
+// Between the passes there are no flags, counters or fences.  The partials start
+// as NaN (the host clears them before the launch) and each is published by a single
+// 8-byte store, so a reader knows a partial is there when it no longer reads NaN.
+// Every CTA merges, for the row block its pass 2 turns to next, the partials of all
+// runs into one offset per row by itself (a 4-warp group does this one row block
+// ahead of the MMAs, off the critical path), always in run order: the result does
+// not depend on who finished first.
+//
+// The row offsets ride in the product itself: the merged offset of a row becomes
+// -off/(2 c kFold) as a sum of three 16-bit numbers, written twice into a 16-element
+// extension of the row in shared memory, and pass 2 appends one more k-step of the
+// MMA that multiplies the extension with a constant tile holding kFold.  The three
 // parts carry 24 (bfloat16) or 33 (float16) significant bits, the products are exact
-// and the accumulator is FP32, so D = w - off/c to FP32 rounding.
+// and the accumulator is FP32, so D = w - off/c to FP32 rounding.  Both 16-byte
+// halves of a row are identical in either tile, so the result does not depend on how
+// the 32-byte swizzle orders them.
 //
 // Each pipeline has its own TMA warp, MMA warp and two 4-warp softmax groups; pass 1
-// never waits on pass 2, so the flag waits of pass 2 cannot deadlock.  The kernel
-// is launched cooperatively with at most one CTA per SM, which guarantees that
-// the CTAs a flag depends on are running.  Every wait is bounded in time; on
+// never waits on pass 2 of another CTA, so the waits of pass 2 cannot deadlock.  The
+// kernel is launched cooperatively with at most one CTA per SM, which guarantees that
+// the CTAs a partial comes from are running.  Every wait is bounded in time; on
 // expiry the kernel records AHAKV_ERR_TIMEOUT in the status word and winds down.
 #include <cuda.h>
 
@@ -41,7 +50,7 @@ namespace {
 
 constexpr int kStages = 2;                 // K-tile ring depth per pipeline
 constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 16-bit elements, 128-byte swizzled
-constexpr int kThreads = 768;              // 4 service warps, 8 + 8 softmax warps, the 4-warp publisher group
+constexpr int kThreads = 768;              // 4 service warps, 8 + 8 softmax warps, the 4-warp merge group
 constexpr long long kWaitLimitNs = 1000000000LL;   // 1 s
 constexpr float kFold = 256.f;             // value of the constant tile; offsets are stored divided by it
 
@@ -56,10 +65,7 @@ struct TcArgs {
   float c[kMaxRows];     // lambda_i log2(e) per observation row
   float cs[128];         // the same per stacked row of a row block (r <= 128 only)
   float2* partial;   // [unit][run][128]
-  uint16_t* qx;      // [unit][128][16] 16-bit: the rows' offset extensions
   float* s_raw;      // [unit][n]
-  int* cnt;          // [unit] partials delivered
-  int* flag;         // [unit] rows whose offset is ready (128 = all)
   int* status;
 };
 
@@ -70,25 +76,24 @@ struct __align__(8) Barriers {
   unsigned long long k_empty[2][kStages];
   unsigned long long acc_full[2][2];
   unsigned long long acc_empty[2][2];
-  unsigned long long pub_full[2];          // row statistics of a run: softmax group -> publisher
-  unsigned long long pub_free[2];
+  unsigned long long ext_full[2];          // offset extension of a row block: merge group -> pass-2 MMA
+  unsigned long long ext_empty[2];
 };
 
 struct Shared {
   Barriers bars;
   uint32_t tmem_slot;
-  int bcast;
   int p2_unit;                  // row block pass 2 of this CTA is working on
   float c[kMaxRows];            // lambda_i * log2(e) per observation row
   float cs2[2][128];            // c per stacked row, by row block parity (r > 128 has two kinds of block)
-  float2 pub[2][256];           // pass 1 (both column halves) -> publisher
+  float2 p1_part[2][128];       // pass 1: statistics of the second half of the key columns
   float p2_part[2][128];        // pass 2: partial column sums of the second half of the rows
 };
 
 constexpr int kQBytes = 2 * kSubTileBytes;              // per pipeline, D <= 128
 constexpr int kKRingBytes = kStages * 2 * kSubTileBytes;
 constexpr int kExtBytes = 128 * 32;                      // 128 rows x 16 16-bit elements, 32-byte swizzled
-constexpr int kSmemTiles = 2 * (kQBytes + kKRingBytes) + 2 * kExtBytes;  // 200 KiB
+constexpr int kSmemTiles = 2 * (kQBytes + kKRingBytes) + 3 * kExtBytes;  // 204 KiB: + two extensions, one constant tile
 constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 8192 /*barriers, constants*/;
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
@@ -138,13 +143,6 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, v
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-      : "memory");
-}
-
-__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
 
@@ -247,10 +245,14 @@ __device__ __forceinline__ void group_sync(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
-__device__ __forceinline__ int ld_acquire(const int* p) {
-  int v;
-  asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+// One partial, straight from L2 (other CTAs write it while this one polls).
+__device__ __forceinline__ float2 ld_partial(const float2* p) {
+  float2 v;
+  asm volatile("ld.relaxed.gpu.global.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
   return v;
+}
+__device__ __forceinline__ void st_partial(float2* p, float2 v) {
+  asm volatile("st.relaxed.gpu.global.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(v.x), "f"(v.y) : "memory");
 }
 
 // ---- work decomposition ----------------------------------------------------------------------------------
@@ -290,8 +292,8 @@ __device__ __forceinline__ int obs_row(const TcArgs& a, const UnitInfo& u, int s
 // ---- roles --------------------------------------------------------------------------------------------
 // TMA producer of one pipeline.  The pass-1 producer also keeps pass 1 from running more than `lag` row
 // blocks ahead of this CTA's pass 2, so that the keys pass 2 re-reads are still in L2.
-__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, const CUtensorMap* xmap,
-                         Shared* sh, int pipe, char* q_smem, char* k_ring, char* ext_smem) {
+__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, Shared* sh, int pipe,
+                         char* q_smem, char* k_ring) {
   Barriers* bars = &sh->bars;
   const int n_sub = a.D / 64;
   const int q_rows = a.r <= 128 ? a.hb * a.r : 128;
@@ -314,27 +316,11 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
       if (!ok) break;
     }
     if (rn.unit != prev_unit) {
-      if (pipe == 1) {
-        // Pass 2 may start on a row block once its statistics are complete: the offset extension of
-        // its rows is then in global memory.
-        *(volatile int*)&sh->p2_unit = rn.unit;              // lets pass 1 move on (see above)
-        const long long t0 = now_ns();
-        while (ld_acquire(&a.flag[rn.unit]) < 128) {
-          __nanosleep(100);
-          if (now_ns() - t0 > kWaitLimitNs) {
-            atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
-            ok = false;
-            break;
-          }
-        }
-        if (!ok) break;
-        asm volatile("fence.proxy.async;" ::: "memory");     // the extension was written with plain stores
-      }
+      if (pipe == 1) *(volatile int*)&sh->p2_unit = rn.unit;   // lets pass 1 move on (see above)
       // the Q buffer is free once every product issued so far has completed
       if (it > 0) ok = mbar_wait(&bars->k_empty[pipe][(it - 1) % kStages], ((it - 1) / kStages) & 1, a.status);
       if (!ok) break;
-      mbar_expect_tx(&bars->q_full[pipe], q_bytes + (pipe == 1 ? kExtBytes : 0));
-      if (pipe == 1) tma_load_3d(ext_smem, xmap, &bars->q_full[pipe], 0, 0, rn.unit);
+      mbar_expect_tx(&bars->q_full[pipe], q_bytes);
       for (int s = 0; s < n_sub; ++s) {
         if (a.r <= 128) tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[pipe], s * 64, 0, u.h * a.G + u.rb * a.hb, u.b);
         else tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[pipe], s * 64, u.rb * 128, u.h, u.b);
@@ -369,10 +355,16 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, int pipe, char* q_smem, 
     const Run rn = run_info(a, run);
     if (rn.unit != prev_unit) {
       if (!mbar_wait(&bars->q_full[pipe], q_loads & 1, a.status)) return;
+      if (pipe == 1) {
+        // the row block's offset extension, from this CTA's merge group
+        if (!mbar_wait(&bars->ext_full[q_loads & 1], (q_loads >> 1) & 1, a.status)) return;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        idesc = umma_idesc(128, unit_info(a, rn.unit).npad, a.bf16);
+      }
       ++q_loads;
       prev_unit = rn.unit;
-      if (pipe == 1) idesc = umma_idesc(128, unit_info(a, rn.unit).npad, a.bf16);
     }
+    const int ext_slot = (q_loads - 1) & 1;
     for (int t = 0; t < rn.cnt; ++t, ++it) {
       const int stage = it % kStages, ph = (it / kStages) & 1, acc = it & 1, aph = (it >> 1) & 1;
       if (!mbar_wait(&bars->acc_empty[pipe][acc], aph ^ 1, a.status)) return;
@@ -387,9 +379,15 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, int pipe, char* q_smem, 
         else umma(d_tmem, kd, qd, idesc, kk > 0);
       }
       // pass 2: D -= off / c, as one more k-step over the constant tile and the rows' offset extensions
-      if (pipe == 1) umma(d_tmem, umma_desc_ext(smem_u32(fold_smem)), umma_desc_ext(smem_u32(ext_smem)), idesc, 1);
+      if (pipe == 1)
+        umma(d_tmem, umma_desc_ext(smem_u32(fold_smem)), umma_desc_ext(smem_u32(ext_smem + ext_slot * kExtBytes)), idesc, 1);
       tc_commit(&bars->k_empty[pipe][stage]);
       tc_commit(&bars->acc_full[pipe][acc]);
+    }
+    if (pipe == 1) {
+      // the extension is free for the merge group once the row block's last product has read it
+      const int next = run + (int)gridDim.x;
+      if (next >= a.n_runs || run_info(a, next).unit != rn.unit) tc_commit(&bars->ext_empty[ext_slot]);
     }
   }
 }
@@ -449,23 +447,24 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
 }
 
 // Pass-1 softmax groups: two groups of four warps share each accumulator; thread `s` of group `half`
-// owns stacked row s over key columns [64 half, 64 half + 64) of the tile.  One (shift, sum) pair per run
-// and half goes to the publisher group through shared memory, so these groups never wait on global memory.
+// owns stacked row s over key columns [64 half, 64 half + 64) of the tile.  At the end of a run group 1
+// hands its (shift, sum) over through shared memory and group 0 publishes the row's partial with one
+// 8-byte store.
 __device__ void row_stats_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int half) {
   Barriers* bars = &sh->bars;
   const int s = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
   int it = 0, run_it = 0;
-  bool dead = false;   // a wait ran out: skip everything that is left
-  for (int run = blockIdx.x; run < a.n_runs && !dead; run += gridDim.x, ++run_it) {
+  bool gone = false;   // a wait ran out: keep only the group barrier
+  for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x, ++run_it) {
     const Run rn = run_info(a, run);
     const UnitInfo u = unit_info(a, rn.unit);
     const int i = obs_row(a, u, s);
     const float c = sh->c[i < a.r ? i : 0];
     const int last = a.n - a.r + i;                       // last visible key of this row
     float M = -INFINITY, Z = 0.f;
-    for (int t = 0; t < rn.cnt; ++t, ++it) {
+    for (int t = 0; t < rn.cnt && !gone; ++t, ++it) {
       const int acc = it & 1, aph = (it >> 1) & 1;
-      if (!mbar_wait(&bars->acc_full[0][acc], aph, a.status)) { dead = true; break; }
+      if (!mbar_wait(&bars->acc_full[0][acc], aph, a.status)) { gone = true; break; }
       tc_fence_after();
       const int j0 = (rn.blk0 + t) * kKeyTile + 64 * half;
       const bool full = (rn.blk0 + t) * kKeyTile + kKeyTile - 1 <= a.n - a.r;   // no key of the tile is masked
@@ -482,93 +481,101 @@ __device__ void row_stats_group(const TcArgs& a, Shared* sh, uint32_t tmem_base,
       mbar_arrive(&bars->acc_empty[0][acc]);               // the accumulator is free for the next product
       fold_chunk(ra, full, j0 + 32, last, c, M, Z);
     }
-    if (dead) break;
-    const int slot = run_it & 1, sph = (run_it >> 1) & 1;
-    if (!mbar_wait(&bars->pub_free[slot], sph ^ 1, a.status)) break;
-    sh->pub[slot][128 * half + s] = make_float2(M, Z);
-    mbar_arrive(&bars->pub_full[slot]);
+    // Both groups meet here once per run, also after a wait has run out, so that nobody is left at the
+    // barrier.  Two slots: group 1 can be at most one run ahead of group 0's read.
+    const int slot = run_it & 1;
+    if (half == 1) sh->p1_part[slot][s] = make_float2(M, Z);
+    group_sync(5, 256);
+    if (half == 0 && !gone) {
+      const float2 e = sh->p1_part[slot][s];
+      const float m = fmaxf(M, e.x);
+      float z = 0.f;
+      if (Z > 0.f) z += Z * fast_exp2(M - m);
+      if (e.y > 0.f) z += e.y * fast_exp2(e.x - m);
+      st_partial(&a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s], make_float2(m, z));
+    }
   }
 }
 
-// Publisher group: moves each run's row statistics to global memory, counts the runs of a row block and,
-// on delivering the last one, merges all of them into one offset per row and raises the block's flag.
-__device__ void publisher_group(const TcArgs& a, Shared* sh) {
+// Merge group: for every row block this CTA's pass 2 turns to, thread `s` waits until the partials of
+// row s have arrived from all runs, merges them in run order into the row's offset and writes the row's
+// offset extension into shared memory for the pass-2 MMA.  It works one row block ahead of the MMA.
+__device__ void merge_group(const TcArgs& a, Shared* sh, char* ext_smem) {
   Barriers* bars = &sh->bars;
   const int s = threadIdx.x & 127;
-  int run_it = 0;
-  bool dead = false;   // a wait ran out: stay in the group's barrier protocol, skip everything else
-  for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x, ++run_it) {
+  int prev_unit = -1, uc = 0;
+  bool dead = false;   // a wait ran out: nothing more is delivered (the MMA warp's own waits then run out too)
+  for (int run = blockIdx.x; run < a.n_runs && !dead; run += gridDim.x) {
     const Run rn = run_info(a, run);
-    const int slot = run_it & 1, sph = (run_it >> 1) & 1;
-    if (!dead && !mbar_wait(&bars->pub_full[slot], sph, a.status)) dead = true;
-    if (!dead) {
-      const float2 e0 = sh->pub[slot][s], e1 = sh->pub[slot][128 + s];   // the two column halves of the row
-      mbar_arrive(&bars->pub_free[slot]);
-      float2 e;
-      e.x = fmaxf(e0.x, e1.x);
-      e.y = (e0.y > 0.f ? e0.y * fast_exp2(e0.x - e.x) : 0.f) + (e1.y > 0.f ? e1.y * fast_exp2(e1.x - e.x) : 0.f);
-      a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s] = e;
-      __threadfence();
-    }
-    group_sync(3, 128);
-    if (s == 0) sh->bcast = dead ? -1 : atomicAdd(&a.cnt[rn.unit], 1);
-    group_sync(3, 128);
-    const bool last_run = sh->bcast == a.rpu - 1;
-    group_sync(3, 128);                                         // bcast may be rewritten after this point
-    if (last_run && !dead) {
-      __threadfence();
-      const float2* p = a.partial + (size_t)rn.unit * a.rpu * 128 + s;
-      float Mx = -INFINITY, Zs = 0.f;
-      for (int t0 = 0; t0 < a.rpu; t0 += 16) {             // 16 loads in flight per thread
-        float2 e[16];
+    if (rn.unit == prev_unit) continue;
+    prev_unit = rn.unit;
+    const UnitInfo u = unit_info(a, rn.unit);
+    const int slot = uc & 1;
+    if (!mbar_wait(&bars->ext_empty[slot], ((uc >> 1) & 1) ^ 1, a.status)) break;
+    ++uc;
+    const float2* p = a.partial + (size_t)rn.unit * a.rpu * 128 + s;
+    float Mx = -INFINITY, Zs = 0.f;
+    for (int t0 = 0; t0 < a.rpu && !dead; t0 += 16) {     // 16 loads in flight per thread
+      float2 e[16];
+      const long long tstart = now_ns();
+      for (;;) {
+        bool all = true;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+          e[t] = t0 + t < a.rpu ? ld_partial(&p[(size_t)(t0 + t) * 128]) : make_float2(-INFINITY, 0.f);
+          all = all && (e[t].x == e[t].x);                 // NaN: not published yet
+        }
+        if (all) break;
+        __nanosleep(200);
+        if (now_ns() - tstart > kWaitLimitNs) {
+          atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
+          dead = true;
+          break;
+        }
+      }
+      if (dead) break;
+      float m = Mx;
+#pragma unroll
+      for (int t = 0; t < 16; ++t) m = fmaxf(m, e[t].x);
+      if (m > -INFINITY) {
+        float z = Zs > 0.f ? Zs * fast_exp2(Mx - m) : 0.f;
 #pragma unroll
         for (int t = 0; t < 16; ++t)
-          e[t] = t0 + t < a.rpu ? __ldcg(&p[(size_t)(t0 + t) * 128]) : make_float2(-INFINITY, 0.f);
-        float m = Mx;
-#pragma unroll
-        for (int t = 0; t < 16; ++t) m = fmaxf(m, e[t].x);
-        if (m > -INFINITY) {
-          float z = Zs > 0.f ? Zs * fast_exp2(Mx - m) : 0.f;
-#pragma unroll
-          for (int t = 0; t < 16; ++t)
-            if (e[t].y > 0.f) z += e[t].y * fast_exp2(e[t].x - m);
-          Zs = z;
-          Mx = m;
-        }
+          if (e[t].y > 0.f) z += e[t].y * fast_exp2(e[t].x - m);
+        Zs = z;
+        Mx = m;
       }
-      // 2^{c w - off} = softmax weight / G.  Pass 2 gets -off / (c kFold) as three 16-bit parts, the
-      // first three of the row's sixteen extension elements; the other thirteen are zero.
-      const UnitInfo u = unit_info(a, rn.unit);
-      uint32_t w0 = 0, w1 = 0;
-      if (s < u.rows) {
-        const float off = Mx + log2f(Zs) + a.log2G;
-        float v = -(off / sh->c[obs_row(a, u, s)]) / kFold;
-        if (a.bf16) {
-          const __nv_bfloat16 h1 = __float2bfloat16_rn(v);
-          v -= __bfloat162float(h1);
-          const __nv_bfloat16 h2 = __float2bfloat16_rn(v);
-          v -= __bfloat162float(h2);
-          const __nv_bfloat16 h3 = __float2bfloat16_rn(v);
-          w0 = (uint32_t)__bfloat16_as_ushort(h1) | ((uint32_t)__bfloat16_as_ushort(h2) << 16);
-          w1 = (uint32_t)__bfloat16_as_ushort(h3);
-        } else {
-          v = fminf(fmaxf(v, -60000.f), 60000.f);            // float16 has no room beyond; such logits are not scored
-          const __half h1 = __float2half_rn(v);
-          v -= __half2float(h1);
-          const __half h2 = __float2half_rn(v);
-          v -= __half2float(h2);
-          const __half h3 = __float2half_rn(v);
-          w0 = (uint32_t)__half_as_ushort(h1) | ((uint32_t)__half_as_ushort(h2) << 16);
-          w1 = (uint32_t)__half_as_ushort(h3);
-        }
-      }
-      uint4* row = reinterpret_cast<uint4*>(a.qx + ((size_t)rn.unit * 128 + s) * 16);
-      row[0] = make_uint4(w0, w1, 0u, 0u);
-      row[1] = make_uint4(0u, 0u, 0u, 0u);
-      __threadfence();
-      asm volatile("fence.proxy.async;" ::: "memory");     // the rows are read back by bulk tensor copies
-      atomicAdd(&a.flag[rn.unit], 1);                      // the block is ready when all 128 rows have reported
     }
+    if (dead) break;
+    // 2^{c w - off} = softmax weight / G.  The MMA adds 2 kFold (h1 + h2 + h3) = -off / c to w.
+    uint32_t w0 = 0, w1 = 0;
+    if (s < u.rows) {
+      const float off = Mx + log2f(Zs) + a.log2G;
+      float v = -(off / sh->c[obs_row(a, u, s)]) / (2.f * kFold);
+      if (a.bf16) {
+        const __nv_bfloat16 h1 = __float2bfloat16_rn(v);
+        v -= __bfloat162float(h1);
+        const __nv_bfloat16 h2 = __float2bfloat16_rn(v);
+        v -= __bfloat162float(h2);
+        const __nv_bfloat16 h3 = __float2bfloat16_rn(v);
+        w0 = (uint32_t)__bfloat16_as_ushort(h1) | ((uint32_t)__bfloat16_as_ushort(h2) << 16);
+        w1 = (uint32_t)__bfloat16_as_ushort(h3);
+      } else {
+        v = fminf(fmaxf(v, -60000.f), 60000.f);            // float16 has no room beyond; such logits are not scored
+        const __half h1 = __float2half_rn(v);
+        v -= __half2float(h1);
+        const __half h2 = __float2half_rn(v);
+        v -= __half2float(h2);
+        const __half h3 = __float2half_rn(v);
+        w0 = (uint32_t)__half_as_ushort(h1) | ((uint32_t)__half_as_ushort(h2) << 16);
+        w1 = (uint32_t)__half_as_ushort(h3);
+      }
+    }
+    uint4* row = reinterpret_cast<uint4*>(ext_smem + slot * kExtBytes + s * 32);
+    row[0] = make_uint4(w0, w1, 0u, 0u);
+    row[1] = make_uint4(w0, w1, 0u, 0u);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads it through the async proxy
+    mbar_arrive(&bars->ext_full[slot]);
   }
 }
 
@@ -656,13 +663,13 @@ __device__ __forceinline__ void column_sum_group(const TcArgs& a, Shared* sh, ui
 
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
-                const __grid_constant__ CUtensorMap xmap, const __grid_constant__ TcArgs a) {
+                const __grid_constant__ TcArgs a) {
   extern __shared__ char smem_raw[];
   char* tiles = reinterpret_cast<char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   char* q_smem[2] = {tiles, tiles + kQBytes + kKRingBytes};
   char* k_ring[2] = {tiles + kQBytes, tiles + 2 * kQBytes + kKRingBytes};
-  char* ext_smem = tiles + 2 * (kQBytes + kKRingBytes);   // pass 2: offset extension of the current rows
-  char* fold_smem = ext_smem + kExtBytes;                 // pass 2: the constant tile
+  char* ext_smem = tiles + 2 * (kQBytes + kKRingBytes);   // pass 2: two offset extensions (current, next)
+  char* fold_smem = ext_smem + 2 * kExtBytes;             // pass 2: the constant tile
   Shared* sh = reinterpret_cast<Shared*>(tiles + kSmemTiles);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -672,8 +679,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     sh->cs2[1][t] = a.r <= 128 ? a.c[t % a.r] : a.c[128 + t];
   }
   {
-    // every 16-byte chunk of the constant tile reads (kFold, kFold, kFold, 0, 0, 0, 0, 0), whatever
-    // the swizzle does to the order of the chunks; it meets the three parts of the rows' extensions
+    // every 16-byte chunk of the constant tile reads (kFold, kFold, kFold, 0, 0, 0, 0, 0); it meets the
+    // three parts of a row's extension twice, once per 16-byte half of the row
     const uint32_t one = a.bf16 ? (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(kFold))
                                 : (uint32_t)__half_as_ushort(__float2half_rn(kFold));
     uint4* f = reinterpret_cast<uint4*>(fold_smem);
@@ -698,11 +705,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
         mbar_init(&bars->acc_full[p][s], 1);
         mbar_init(&bars->acc_empty[p][s], 256);
       }
-      mbar_init(&bars->pub_full[p], 256);
-      mbar_init(&bars->pub_free[p], 128);
+      mbar_init(&bars->ext_full[p], 128);
+      mbar_init(&bars->ext_empty[p], 1);
     }
     sh->p2_unit = 0;
-    sh->bcast = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // all 512 TMEM columns: four 128-column accumulators
@@ -715,11 +721,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   const uint32_t tmem_base = sh->tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) producer(a, &qmap, &kmap, &xmap, sh, 0, q_smem[0], k_ring[0], ext_smem);
+    if (lane == 0) producer(a, &qmap, &kmap, sh, 0, q_smem[0], k_ring[0]);
   } else if (warp == 1) {
     if (lane == 0) mma_issuer(a, sh, 0, q_smem[0], k_ring[0], ext_smem, fold_smem, tmem_base);
   } else if (warp == 2) {
-    if (lane == 0) producer(a, &qmap, &kmap, &xmap, sh, 1, q_smem[1], k_ring[1], ext_smem);
+    if (lane == 0) producer(a, &qmap, &kmap, sh, 1, q_smem[1], k_ring[1]);
   } else if (warp == 3) {
     if (lane == 0) mma_issuer(a, sh, 1, q_smem[1], k_ring[1], ext_smem, fold_smem, tmem_base);
   } else if (warp < 12) {
@@ -727,7 +733,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   } else if (warp < 20) {
     column_sum_group(a, sh, tmem_base, (warp - 12) >> 2);
   } else {
-    publisher_group(a, sh);
+    merge_group(a, sh, ext_smem);
   }
 
   tc_fence_before();
@@ -769,24 +775,12 @@ bool make_map(CUtensorMap* m, const void* base, int bf16, int d, long long token
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 3-D map {16, 128, units} over the rows' offset extensions, one {16, 128, 1} box per row block, 32-byte swizzle.
-bool make_ext_map(CUtensorMap* m, const void* base, int bf16, long long units) {
-  const cuuint64_t dims[3] = {16, 128, (cuuint64_t)units};
-  const cuuint64_t strides[2] = {32, 128 * 32};
-  const cuuint32_t box[3] = {16, 128, 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return encode_fn()(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3,
-                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 bool score_tc_available() { return encode_fn() != nullptr; }
 
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float* s_raw, float2* partial,
-                             void* row_ext, int* sync_words, int* status, cudaStream_t st) {
+                             int* status, cudaStream_t st) {
   static int n_sm = 0;
   static bool configured = false;
   if (!configured) {
@@ -814,18 +808,19 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float
   a.log2G = log2f((float)pl.G);
   for (int i = 0; i < kMaxRows; ++i) a.c[i] = pl.rows.c[i];
   for (int t = 0; t < 128; ++t) a.cs[t] = pl.r <= 128 ? pl.rows.c[t % pl.r] : 0.f;
-  a.partial = partial; a.qx = static_cast<uint16_t*>(row_ext); a.s_raw = s_raw;
-  a.cnt = sync_words; a.flag = sync_words + units; a.status = status;
+  a.partial = partial; a.s_raw = s_raw;
+  a.status = status;
 
-  CUtensorMap qmap, kmap, xmap;
+  CUtensorMap qmap, kmap;
   const int q_box_rows = pl.r <= 128 ? pl.r : 128, q_box_heads = pl.r <= 128 ? pl.heads_per_rb : 1;
   if (!make_map(&qmap, q, a.bf16, pl.d, pl.r, pl.Hq, pl.B, pl.qs, pl.es, q_box_rows, q_box_heads) ||
-      !make_map(&kmap, k, a.bf16, pl.d, pl.n, pl.Hkv, pl.B, pl.ks, pl.es, kKeyTile, 1) ||
-      !make_ext_map(&xmap, row_ext, a.bf16, units))
+      !make_map(&kmap, k, a.bf16, pl.d, pl.n, pl.Hkv, pl.B, pl.ks, pl.es, kKeyTile, 1))
     return AHAKV_ERR_CUDA;
 
+  // every partial starts as NaN: "not published yet"
+  if (cudaMemsetAsync(partial, 0xff, (size_t)a.n_runs * 128 * sizeof(float2), st) != cudaSuccess) return AHAKV_ERR_CUDA;
   const int grid = a.n_runs < n_sm ? a.n_runs : n_sm;
-  void* args[] = {&qmap, &kmap, &xmap, &a};
+  void* args[] = {&qmap, &kmap, &a};
   const cudaError_t e = cudaLaunchCooperativeKernel((const void*)score_tc_kernel, dim3(grid), dim3(kThreads), args,
                                                     (size_t)kSmemBytes, st);
   count_launch();
