@@ -797,12 +797,12 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float
   a.n_blk = pl.n_blk; a.D = pl.d;
   const long long tiles = (long long)units * pl.n_blk;
   const long long ch = tiles / ((long long)n_sm * 8);
-  a.CH = ch < 1 ? 1 : (ch > 4 ? 4 : (int)ch);
+  a.CH = ch < 1 ? 1 : (ch > 8 ? 8 : (int)ch);
   a.rpu = (pl.n_blk + a.CH - 1) / a.CH;
   a.n_runs = units * a.rpu;
-  // keep about 64 MiB of keys between the two passes: half of L2
+  // keep about 48 MiB of keys between the two passes, which L2 still holds next to the rest of the traffic
   const long long unit_bytes = (long long)pl.n * pl.d * pl.es;
-  const long long lag = (64LL << 20) / (unit_bytes * pl.n_rb > 0 ? unit_bytes : 1) * pl.n_rb;
+  const long long lag = (48LL << 20) / (unit_bytes * pl.n_rb > 0 ? unit_bytes : 1) * pl.n_rb;
   a.lag = lag < 2 * pl.n_rb ? 2 * pl.n_rb : (lag > 4096 ? 4096 : (int)lag);
   a.bf16 = pl.dtype == AHAKV_BF16;
   a.log2G = log2f((float)pl.G);
