@@ -137,6 +137,33 @@ ahakv_status ahakv_profile_enable(int on);
 int64_t ahakv_profile_read(double* ms);
 const char* ahakv_stage_name(int stage);
 
+/* The eviction score for callers that cannot provide scratch memory (this entry point has no
+ * counterpart in the paper; it exists for deployment).  Some users of this library cannot allocate
+ * device memory where they call it: an inference server whose memory pool was sized at start-up and
+ * hands out nothing afterwards, an extension that receives tensors but no allocator, a caller that must
+ * not touch cudaMalloc because it synchronises the device and can fail under memory pressure.  For them
+ * the library carries its own scratch: a device array of AHAKV_STATIC_WS_BYTES that every GPU holds from
+ * the time the library is loaded until the process ends.
+ *
+ * Computes exactly what ahakv_score computes, with the same kernels; the caller passes inputs and
+ * outputs only.  Nothing is allocated or freed, by this call or by anything it calls.
+ *  - Limit: ahakv_workspace_bytes(p) must not exceed AHAKV_STATIC_WS_BYTES (ahakv_static_workspace_bytes()
+ *    returns it at run time); larger problems get AHAKV_ERR_WORKSPACE and nothing is launched.  8 MiB
+ *    covers, for instance, one sequence of 8 KV heads x 16384 tokens (3.5 MiB), 32 heads x 4096 tokens
+ *    (2 MiB) or a 16-sequence decode round of 8 KV heads x 2080 tokens (5.3 MiB); 32 heads x 16384
+ *    tokens (8.02 MiB) is just over.
+ *  - The first call on each device looks up the array's device address (the device must be current, as
+ *    for every other call); make that first call before you start capturing a stream.
+ *  - All calls on a device share the one array, which keeps whatever the last call left in it.  The call
+ *    resets what has to start clean, so calls in sequence are independent; two calls that overlap on the
+ *    GPU (different streams) race on the array and must be serialised by the caller.
+ *  - ahakv_last_device_status cannot be asked about this scratch; a device-side timeout leaves the output
+ *    undefined, exactly as in ahakv_score. */
+#define AHAKV_STATIC_WS_BYTES (8u << 20)
+size_t ahakv_static_workspace_bytes(void);
+ahakv_status ahakv_score_static(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
+                                const float* score_prev, float* score, ahakv_stream_t stream);
+
 /* Number of kernels the library has launched in this process since it was loaded. */
 int64_t ahakv_launch_count(void);
 

@@ -86,6 +86,8 @@ SIGNATURES = {
     "ahakv_select": (ctypes.c_int, [_PP, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_compact": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_evict": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_score_static": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "ahakv_static_workspace_bytes": (_sz, []),
     "ahakv_last_device_status": (ctypes.c_int, [_vp, _vp]),
     "ahakv_launch_count": (ctypes.c_int64, []),
     "ahakv_profile_enable": (ctypes.c_int, [ctypes.c_int]),
@@ -157,6 +159,20 @@ def ahakv_score(p: Params, q_obs, k, v, score_prev, score, ws, ws_bytes: int | N
                            _ptr(ws), nbytes, _stream(stream))
     if check:
         _raise(st, "ahakv_score")
+    return st
+
+
+def ahakv_static_workspace_bytes() -> int:
+    return int(lib().ahakv_static_workspace_bytes())
+
+
+def ahakv_score_static(p: Params, q_obs, k, v, score_prev, score, stream=None, check: bool = True) -> int:
+    """``ahakv_score`` on the library's own fixed scratch array: no workspace argument, no allocation."""
+    cp = p.c()
+    st = lib().ahakv_score_static(ctypes.byref(cp), _ptr(q_obs), _ptr(k), _ptr(v), _ptr(score_prev),
+                                  _ptr(score), _stream(stream))
+    if check:
+        _raise(st, "ahakv_score_static")
     return st
 
 
