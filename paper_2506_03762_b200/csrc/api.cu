@@ -130,15 +130,15 @@ static ahakv_status queue_score(const Plan& pl, const void* q, const void* k, co
   float* s_raw = at<float>(ws, pl.off_sraw);
   float2* partial = at<float2>(ws, pl.off_partial);
   float* final_off = at<float>(ws, pl.off_final);
-  if (pl.use_tc)
-    rc = launch_score_tc(pl, q, k, s_raw, partial, at<int>(ws, pl.off_status), st);
+  const bool prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0;
+  float* nu = prior ? at<float>(ws, pl.off_nu) : nullptr;
+  if (pl.use_tc)   // the tensor-core kernel squares the value rows on its way
+    rc = launch_score_tc(pl, q, k, prior ? v : nullptr, s_raw, nu, partial, at<int>(ws, pl.off_status), st);
   else
     rc = launch_score_simt(pl, q, k, s_raw, partial, final_off, st);
   if (rc) return rc;
   profile_mark(prof, 1, st);
-  float* nu = nullptr;
-  if (pl.flags & AHAKV_FLAG_VALUE_PRIOR) {
-    nu = at<float>(ws, pl.off_nu);
+  if (prior && !pl.use_tc) {
     rc = launch_vnorm(pl, v, nu, st);
     if (rc) return rc;
   }

@@ -1,11 +1,11 @@
 // Tensor-core scoring for 16-bit inputs on sm_100a: one persistent kernel that
-// computes the accumulated SG-softmax score (Eq. 1, 5, 9) of every KV head.
+// computes the accumulated SG-softmax score (Eq. 1, 5, 9) of every KV head and,
+// on the way, the squared value norms of Section 4.3.
 //
 // Work unit: a "row block" = up to 128 stacked observation rows (query heads of
 // one KV head x observation rows) against all n keys, cut into 128-key tiles.
 // A normalised column sum needs each row's softmax statistics over ALL keys
-// first, so every tile is visited twice, by two pipelines that live side by side
-// in each CTA and share nothing but the SM:
+// first, so every tile is visited twice:
 //
 //   pass 1 (rows on TMEM lanes):  D = Q . K^T   -> per-row (shift, sum of 2^{c w - shift})
 //                                 of a run of tiles, stored to global memory as one
@@ -16,16 +16,24 @@
 //
 // Both products are tcgen05.mma kind::f16 with FP32 accumulators in TMEM, fed by
 // TMA (128-byte swizzle) from the same K-major Q and K tiles, which serve as A or
-// B operand alike.  Pass 2 trails pass 1 by a few row blocks, so its second read
-// of K is served by L2 and HBM sees K once.
+// B operand alike.
+//
+// Schedule.  A run is up to CH consecutive key tiles of one row block; run q belongs
+// to CTA q mod grid.  Every CTA walks ONE fixed sequence of segments,
+//     P1(run 0) .. P1(run lead-1), then P1(run i+lead), P2(run i), P1(run i+lead+1), P2(run i+1), ..
+// through one pipeline: one TMA warp, one MMA warp, a ring of K tiles, four TMEM
+// accumulators and sixteen softmax warps that take whichever kind of tile comes
+// next.  Pass 2 of a run thus trails its pass 1 by `lead` steps: long enough for
+// every CTA to have delivered its share of the row block's statistics, short
+// enough for the keys to be still in L2, so that HBM sees K once.
 //
 // Between the passes there are no flags, counters or fences.  The partials start
 // as NaN (the host clears them before the launch) and each is published by a single
 // 8-byte store, so a reader knows a partial is there when it no longer reads NaN.
-// Every CTA merges, for the row block its pass 2 turns to next, the partials of all
-// runs into one offset per row by itself (a 4-warp group does this one row block
-// ahead of the MMAs, off the critical path), always in run order: the result does
-// not depend on who finished first.
+// Every CTA merges, for the run its pass 2 turns to next, the partials of all
+// runs of that row block into one offset per row by itself (a 4-warp group does this
+// one step ahead of the MMAs, off the critical path), always in run order: the
+// result does not depend on who finished first.
 //
 // The row offsets ride in the product itself: the merged offset of a row becomes
 // -off/(2 c kFold) as a sum of three 16-bit numbers, written twice into a 16-element
@@ -36,11 +44,15 @@
 // halves of a row are identical in either tile, so the result does not depend on how
 // the 32-byte swizzle orders them.
 //
-// Each pipeline has its own TMA warp, MMA warp and two 4-warp softmax groups; pass 1
-// never waits on pass 2 of another CTA, so the waits of pass 2 cannot deadlock.  The
-// kernel is launched cooperatively with at most one CTA per SM, which guarantees that
-// the CTAs a partial comes from are running.  Every wait is bounded in time; on
-// expiry the kernel records AHAKV_ERR_TIMEOUT in the status word and winds down.
+// The value rows of the keys of each pass-1 tile stream through a small ring of their
+// own (a second TMA warp, evict-first in L2) and the same 4-warp group squares and
+// adds them: nu_j = |V_j|^2 costs no launch and no second sweep of HBM.
+//
+// The kernel is launched cooperatively with at most one CTA per SM, which guarantees
+// that the CTAs a partial comes from are running; a wait only ever depends on work
+// that is earlier in the fixed sequence, so the waits cannot deadlock.  Every wait is
+// bounded in time; on expiry the kernel records AHAKV_ERR_TIMEOUT in the status word
+// and winds down.
 #include <cuda.h>
 
 #include "ahakv_internal.cuh"
@@ -48,9 +60,11 @@
 namespace ahakv {
 namespace {
 
-constexpr int kStages = 2;                 // K-tile ring depth per pipeline
+constexpr int kKStages = 3;                // K-tile ring depth
 constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 16-bit elements, 128-byte swizzled
-constexpr int kThreads = 768;              // 4 service warps, 8 + 8 softmax warps, the 4-warp merge group
+constexpr int kVRows = 64;                 // value rows per V-ring stage
+constexpr int kVSubBytes = kVRows * 128;
+constexpr int kThreads = 768;              // 4 service warps, 16 softmax warps, the 4-warp merge / value-norm group
 constexpr long long kWaitLimitNs = 1000000000LL;   // 1 s
 constexpr float kFold = 256.f;             // value of the constant tile; offsets are stored divided by it
 
@@ -59,42 +73,48 @@ struct TcArgs {
   int CH;         // key tiles per run
   int rpu;        // runs per row block = ceil(n_blk / CH)
   int n_runs;     // row blocks * rpu
-  int lag;        // pass 1 may lead this CTA's pass 2 by at most this many row blocks
+  int lead;       // pass 2 of a run comes `lead` steps after its pass 1
   int bf16;       // operand type of the products
+  int prior;      // stream V and write nu
   float log2G;
   float c[kMaxRows];     // lambda_i log2(e) per observation row
   float cs[128];         // the same per stacked row of a row block (r <= 128 only)
   float2* partial;   // [unit][run][128]
   float* s_raw;      // [unit][n]
+  float* nu;         // [B * Hkv][n]
   int* status;
 };
 
 // ---- shared memory layout --------------------------------------------------------------------
 struct __align__(8) Barriers {
-  unsigned long long q_full[2];            // [pipeline]
-  unsigned long long k_full[2][kStages];
-  unsigned long long k_empty[2][kStages];
-  unsigned long long acc_full[2][2];
-  unsigned long long acc_empty[2][2];
-  unsigned long long ext_full[2];          // offset extension of a row block: merge group -> pass-2 MMA
-  unsigned long long ext_empty[2];
+  unsigned long long q_full[2], q_empty[2];
+  unsigned long long k_full[kKStages], k_empty[kKStages];
+  unsigned long long v_full[2], v_empty[2];
+  unsigned long long acc_full[4], acc_empty[4];
+  unsigned long long ext_full[2], ext_empty[2];   // offset extension of a run's row block: merge group -> MMA
 };
 
 struct Shared {
   Barriers bars;
   uint32_t tmem_slot;
-  int p2_unit;                  // row block pass 2 of this CTA is working on
+  int pad_;
   float c[kMaxRows];            // lambda_i * log2(e) per observation row
   float cs2[2][128];            // c per stacked row, by row block parity (r > 128 has two kinds of block)
-  float2 p1_part[2][128];       // pass 1: statistics of the second half of the key columns
-  float p2_part[2][128];        // pass 2: partial column sums of the second half of the rows
+  float2 p1_part[2][3][128];    // pass 1: statistics of the three groups that do not publish
+  float p2_part[2][2][128];     // pass 2: partial column sums of the second half of the rows, per pair
 };
 
-constexpr int kQBytes = 2 * kSubTileBytes;              // per pipeline, D <= 128
-constexpr int kKRingBytes = kStages * 2 * kSubTileBytes;
+constexpr int kQBytes = 2 * kSubTileBytes;              // D <= 128
+constexpr int kKStageBytes = 2 * kSubTileBytes;
+constexpr int kVStageBytes = 2 * kVSubBytes;
 constexpr int kExtBytes = 128 * 32;                      // 128 rows x 16 16-bit elements, 32-byte swizzled
-constexpr int kSmemTiles = 2 * (kQBytes + kKRingBytes) + 3 * kExtBytes;  // 204 KiB: + two extensions, one constant tile
-constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 8192 /*barriers, constants*/;
+constexpr int kOffQ = 0;
+constexpr int kOffK = kOffQ + 2 * kQBytes;
+constexpr int kOffV = kOffK + kKStages * kKStageBytes;
+constexpr int kOffExt = kOffV + 2 * kVStageBytes;        // two extensions, then the constant tile
+constexpr int kSmemTiles = kOffExt + 3 * kExtBytes;      // 204 KiB
+constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 12288 /*barriers, constants, exchange*/;
+static_assert(sizeof(Shared) <= 12288, "Shared outgrew its reservation");
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -289,55 +309,67 @@ __device__ __forceinline__ int obs_row(const TcArgs& a, const UnitInfo& u, int s
   return a.r <= 128 ? s % a.r : u.rb * 128 + s;
 }
 
+__device__ __forceinline__ void tma_load_4d_hint(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2,
+                                                 int c3, unsigned long long policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ unsigned long long policy_evict_first() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+
+// The fixed sequence of segments of this CTA: f(pass, run) for P1(0) .. P1(lead-1), then alternately
+// P1(i + lead), P2(i).  Every role walks it with the same counters.
+template <typename F>
+__device__ __forceinline__ void for_each_segment(const TcArgs& a, F f) {
+  const int G = (int)gridDim.x, first = (int)blockIdx.x;
+  const int nr = (a.n_runs - first + G - 1) / G;
+  for (int k = 0; k < nr + a.lead; ++k) {
+    if (k < nr) f(0, first + k * G);
+    if (k >= a.lead) f(1, first + (k - a.lead) * G);
+  }
+}
+
 // ---- roles --------------------------------------------------------------------------------------------
-// TMA producer of one pipeline.  The pass-1 producer also keeps pass 1 from running more than `lag` row
-// blocks ahead of this CTA's pass 2, so that the keys pass 2 re-reads are still in L2.
-__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, Shared* sh, int pipe,
-                         char* q_smem, char* k_ring) {
+// TMA producer of Q and K tiles.
+__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, Shared* sh, char* tiles) {
   Barriers* bars = &sh->bars;
   const int n_sub = a.D / 64;
   const int q_rows = a.r <= 128 ? a.hb * a.r : 128;
   const int q_bytes = n_sub * q_rows * 128, k_bytes = n_sub * kSubTileBytes;
-  int it = 0, prev_unit = -1;
+  const unsigned long long once = policy_evict_first();
+  int tc = 0, sc = 0;
   bool ok = true;
-  for (int run = blockIdx.x; run < a.n_runs && ok; run += gridDim.x) {
+  for_each_segment(a, [&](int pass, int run) {
+    if (!ok) return;
     const Run rn = run_info(a, run);
     const UnitInfo u = unit_info(a, rn.unit);
-    if (pipe == 0 && rn.unit > *(volatile int*)&sh->p2_unit + a.lag) {
-      const long long t0 = now_ns();
-      while (rn.unit > *(volatile int*)&sh->p2_unit + a.lag) {
-        __nanosleep(100);
-        if (now_ns() - t0 > kWaitLimitNs) {
-          atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
-          ok = false;
-          break;
-        }
-      }
-      if (!ok) break;
+    const int qb = sc & 1;
+    char* q_smem = tiles + kOffQ + qb * kQBytes;
+    if (!(ok = mbar_wait(&bars->q_empty[qb], ((sc >> 1) & 1) ^ 1, a.status))) return;
+    mbar_expect_tx(&bars->q_full[qb], q_bytes);
+    for (int s = 0; s < n_sub; ++s) {
+      if (a.r <= 128) tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, 0, u.h * a.G + u.rb * a.hb, u.b);
+      else tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, u.rb * 128, u.h, u.b);
     }
-    if (rn.unit != prev_unit) {
-      if (pipe == 1) *(volatile int*)&sh->p2_unit = rn.unit;   // lets pass 1 move on (see above)
-      // the Q buffer is free once every product issued so far has completed
-      if (it > 0) ok = mbar_wait(&bars->k_empty[pipe][(it - 1) % kStages], ((it - 1) / kStages) & 1, a.status);
-      if (!ok) break;
-      mbar_expect_tx(&bars->q_full[pipe], q_bytes);
+    ++sc;
+    for (int t = 0; t < rn.cnt; ++t, ++tc) {
+      const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
+      if (!(ok = mbar_wait(&bars->k_empty[stage], ph ^ 1, a.status))) return;
+      mbar_expect_tx(&bars->k_full[stage], k_bytes);
+      char* dst = tiles + kOffK + stage * kKStageBytes;
       for (int s = 0; s < n_sub; ++s) {
-        if (a.r <= 128) tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[pipe], s * 64, 0, u.h * a.G + u.rb * a.hb, u.b);
-        else tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[pipe], s * 64, u.rb * 128, u.h, u.b);
+        // the second read of a key tile is its last: let L2 drop it first
+        if (pass == 0) tma_load_4d(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b);
+        else tma_load_4d_hint(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b, once);
       }
-      prev_unit = rn.unit;
     }
-    for (int t = 0; t < rn.cnt && ok; ++t, ++it) {
-      const int stage = it % kStages, ph = (it / kStages) & 1;
-      ok = mbar_wait(&bars->k_empty[pipe][stage], ph ^ 1, a.status);
-      if (!ok) break;
-      mbar_expect_tx(&bars->k_full[pipe][stage], k_bytes);
-      for (int s = 0; s < n_sub; ++s)
-        tma_load_4d(k_ring + (stage * 2 + s) * kSubTileBytes, kmap, &bars->k_full[pipe][stage], s * 64,
-                    (rn.blk0 + t) * kKeyTile, u.h, u.b);
-    }
-  }
-  if (pipe == 1) *(volatile int*)&sh->p2_unit = 0x3fffffff;   // nothing left for pass 1 to wait for
+  });
   if (!ok) {
     // wind down: give copies already in flight a bounded time (1 ms) to land before the CTA exits
     const long long t0 = now_ns();
@@ -345,51 +377,82 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
   }
 }
 
-// MMA issuer of one pipeline.  pipe 0: D[rows x keys] = Q K^T.  pipe 1: D[keys x rows] = K Q^T.
-__device__ void mma_issuer(const TcArgs& a, Shared* sh, int pipe, char* q_smem, char* k_ring, char* ext_smem,
-                           char* fold_smem, uint32_t tmem_base) {
+// TMA producer of the value rows that go with the key tiles of pass 1 (first row block of a KV head only).
+__device__ void v_producer(const TcArgs& a, const CUtensorMap* vmap, Shared* sh, char* tiles) {
   Barriers* bars = &sh->bars;
-  int it = 0, prev_unit = -1, q_loads = 0;
-  uint32_t idesc = umma_idesc(128, 128, a.bf16);
-  for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x) {
+  const int n_sub = a.D / 64;
+  const unsigned long long once = policy_evict_first();
+  int vc = 0;
+  bool ok = true;
+  for_each_segment(a, [&](int pass, int run) {
+    if (pass != 0 || !ok) return;
     const Run rn = run_info(a, run);
-    if (rn.unit != prev_unit) {
-      if (!mbar_wait(&bars->q_full[pipe], q_loads & 1, a.status)) return;
-      if (pipe == 1) {
-        // the row block's offset extension, from this CTA's merge group
-        if (!mbar_wait(&bars->ext_full[q_loads & 1], (q_loads >> 1) & 1, a.status)) return;
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        idesc = umma_idesc(128, unit_info(a, rn.unit).npad, a.bf16);
-      }
-      ++q_loads;
-      prev_unit = rn.unit;
+    const UnitInfo u = unit_info(a, rn.unit);
+    if (u.rb != 0) return;
+    for (int t = 0; t < 2 * rn.cnt; ++t, ++vc) {
+      const int vs = vc & 1;
+      if (!(ok = mbar_wait(&bars->v_empty[vs], ((vc >> 1) & 1) ^ 1, a.status))) return;
+      mbar_expect_tx(&bars->v_full[vs], n_sub * kVSubBytes);
+      char* dst = tiles + kOffV + vs * kVStageBytes;
+      for (int s = 0; s < n_sub; ++s)
+        tma_load_4d_hint(dst + s * kVSubBytes, vmap, &bars->v_full[vs], s * 64, rn.blk0 * kKeyTile + t * kVRows, u.h, u.b, once);
     }
-    const int ext_slot = (q_loads - 1) & 1;
-    for (int t = 0; t < rn.cnt; ++t, ++it) {
-      const int stage = it % kStages, ph = (it / kStages) & 1, acc = it & 1, aph = (it >> 1) & 1;
-      if (!mbar_wait(&bars->acc_empty[pipe][acc], aph ^ 1, a.status)) return;
-      if (!mbar_wait(&bars->k_full[pipe][stage], ph, a.status)) return;
+  });
+  if (!ok) {
+    const long long t0 = now_ns();
+    while (now_ns() - t0 < 1000000) __nanosleep(1000);
+  }
+}
+
+// MMA issuer.  Pass 1: D[rows x keys] = Q K^T.  Pass 2: D[keys x rows] = K Q^T - off / c.
+__device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tmem_base) {
+  Barriers* bars = &sh->bars;
+  int tc = 0, sc = 0, pc = 0;
+  bool ok = true;
+  const uint64_t fold_desc = umma_desc_ext(smem_u32(tiles + kOffExt + 2 * kExtBytes));
+  for_each_segment(a, [&](int pass, int run) {
+    if (!ok) return;
+    const Run rn = run_info(a, run);
+    const int qb = sc & 1;
+    char* q_smem = tiles + kOffQ + qb * kQBytes;
+    if (!(ok = mbar_wait(&bars->q_full[qb], (sc >> 1) & 1, a.status))) return;
+    uint32_t idesc = umma_idesc(128, 128, a.bf16);
+    uint64_t ext_desc = 0;
+    const int slot = pc & 1;
+    if (pass == 1) {
+      // the row block's offset extension, from this CTA's merge group
+      if (!(ok = mbar_wait(&bars->ext_full[slot], (pc >> 1) & 1, a.status))) return;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      idesc = umma_idesc(128, unit_info(a, rn.unit).npad, a.bf16);
+      ext_desc = umma_desc_ext(smem_u32(tiles + kOffExt + slot * kExtBytes));
+    }
+    for (int t = 0; t < rn.cnt; ++t, ++tc) {
+      const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
+      const int acc = (tc & 1) * 2 + ((tc >> 1) & 1), aph = (tc >> 2) & 1;
+      if (!(ok = mbar_wait(&bars->acc_empty[acc], aph ^ 1, a.status))) return;
+      if (!(ok = mbar_wait(&bars->k_full[stage], ph, a.status))) return;
       tc_fence_after();
-      const uint32_t d_tmem = tmem_base + (uint32_t)((pipe * 2 + acc) * 128);
+      const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 128);
+      char* k_smem = tiles + kOffK + stage * kKStageBytes;
       for (int kk = 0; kk < a.D / 16; ++kk) {
         const int sub = kk >> 2, koff = (kk & 3) * 32;
         const uint64_t qd = umma_desc(smem_u32(q_smem + sub * kSubTileBytes) + koff);
-        const uint64_t kd = umma_desc(smem_u32(k_ring + (stage * 2 + sub) * kSubTileBytes) + koff);
-        if (pipe == 0) umma(d_tmem, qd, kd, idesc, kk > 0);
+        const uint64_t kd = umma_desc(smem_u32(k_smem + sub * kSubTileBytes) + koff);
+        if (pass == 0) umma(d_tmem, qd, kd, idesc, kk > 0);
         else umma(d_tmem, kd, qd, idesc, kk > 0);
       }
       // pass 2: D -= off / c, as one more k-step over the constant tile and the rows' offset extensions
-      if (pipe == 1)
-        umma(d_tmem, umma_desc_ext(smem_u32(fold_smem)), umma_desc_ext(smem_u32(ext_smem + ext_slot * kExtBytes)), idesc, 1);
-      tc_commit(&bars->k_empty[pipe][stage]);
-      tc_commit(&bars->acc_full[pipe][acc]);
+      if (pass == 1) umma(d_tmem, fold_desc, ext_desc, idesc, 1);
+      tc_commit(&bars->k_empty[stage]);
+      tc_commit(&bars->acc_full[acc]);
     }
-    if (pipe == 1) {
-      // the extension is free for the merge group once the row block's last product has read it
-      const int next = run + (int)gridDim.x;
-      if (next >= a.n_runs || run_info(a, next).unit != rn.unit) tc_commit(&bars->ext_empty[ext_slot]);
+    tc_commit(&bars->q_empty[qb]);          // Q (and the extension) are free once the segment's products are done
+    if (pass == 1) {
+      tc_commit(&bars->ext_empty[slot]);
+      ++pc;
     }
-  }
+    ++sc;
+  });
 }
 
 // One 32-key chunk of a row: fold it into the running pair (M, Z) with Z = sum of 2^{c w - M}.
@@ -446,73 +509,199 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
   }
 }
 
-// Pass-1 softmax groups: two groups of four warps share each accumulator; thread `s` of group `half`
-// owns stacked row s over key columns [64 half, 64 half + 64) of the tile.  At the end of a run group 1
-// hands its (shift, sum) over through shared memory and group 0 publishes the row's partial with one
-// 8-byte store.
-__device__ void row_stats_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int half) {
-  Barriers* bars = &sh->bars;
-  const int s = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
-  int it = 0, run_it = 0;
-  bool gone = false;   // a wait ran out: keep only the group barrier
-  for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x, ++run_it) {
-    const Run rn = run_info(a, run);
-    const UnitInfo u = unit_info(a, rn.unit);
-    const int i = obs_row(a, u, s);
-    const float c = sh->c[i < a.r ? i : 0];
-    const int last = a.n - a.r + i;                       // last visible key of this row
-    float M = -INFINITY, Z = 0.f;
-    for (int t = 0; t < rn.cnt && !gone; ++t, ++it) {
-      const int acc = it & 1, aph = (it >> 1) & 1;
-      if (!mbar_wait(&bars->acc_full[0][acc], aph, a.status)) { gone = true; break; }
-      tc_fence_after();
-      const int j0 = (rn.blk0 + t) * kKeyTile + 64 * half;
-      const bool full = (rn.blk0 + t) * kKeyTile + kKeyTile - 1 <= a.n - a.r;   // no key of the tile is masked
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 128 + 64 * half);
-      uint32_t ra[32];
-      // One chunk at a time: load, wait, fold.  The other warps of the scheduler fill the load latency;
-      // keeping a second load in flight costs registers and ties the exponentials to its completion.
-      tmem_ld32_issue(taddr, ra);
-      tmem_ld_wait(ra);
-      fold_chunk(ra, full, j0, last, c, M, Z);
-      tmem_ld32_issue(taddr + 32, ra);
-      tmem_ld_wait(ra);
-      tc_fence_before();
-      mbar_arrive(&bars->acc_empty[0][acc]);               // the accumulator is free for the next product
-      fold_chunk(ra, full, j0 + 32, last, c, M, Z);
-    }
-    // Both groups meet here once per run, also after a wait has run out, so that nobody is left at the
-    // barrier.  Two slots: group 1 can be at most one run ahead of group 0's read.
-    const int slot = run_it & 1;
-    if (half == 1) sh->p1_part[slot][s] = make_float2(M, Z);
-    group_sync(5, 256);
-    if (half == 0 && !gone) {
-      const float2 e = sh->p1_part[slot][s];
-      const float m = fmaxf(M, e.x);
-      float z = 0.f;
-      if (Z > 0.f) z += Z * fast_exp2(M - m);
-      if (e.y > 0.f) z += e.y * fast_exp2(e.x - m);
-      st_partial(&a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s], make_float2(m, z));
+// Sixty-four stacked rows of a key's column, rows [64 HALF, 64 HALF + 64): adds 2^{c D} of each.  The
+// column indices are compile-time constants, so every c comes straight from the kernel's parameter
+// bank as an operand of the multiply.
+template <int HALF>
+__device__ __forceinline__ float column_sum_fast(const TcArgs& a, uint32_t taddr) {
+  float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint32_t r[16];
+    tmem_ld16_issue(taddr + 64 * HALF + 16 * q, r);
+    tmem_ld_wait16(r);
+#pragma unroll
+    for (int t = 0; t < 16; t += 4) {
+      z0 += fast_exp2(__uint_as_float(r[t]) * a.cs[64 * HALF + 16 * q + t]);
+      z1 += fast_exp2(__uint_as_float(r[t + 1]) * a.cs[64 * HALF + 16 * q + t + 1]);
+      z2 += fast_exp2(__uint_as_float(r[t + 2]) * a.cs[64 * HALF + 16 * q + t + 2]);
+      z3 += fast_exp2(__uint_as_float(r[t + 3]) * a.cs[64 * HALF + 16 * q + t + 3]);
     }
   }
+  return (z0 + z1) + (z2 + z3);
 }
 
-// Merge group: for every row block this CTA's pass 2 turns to, thread `s` waits until the partials of
-// row s have arrived from all runs, merges them in run order into the row's offset and writes the row's
-// offset extension into shared memory for the pass-2 MMA.  It works one row block ahead of the MMA.
-__device__ void merge_group(const TcArgs& a, Shared* sh, char* ext_smem) {
+// Softmax warps: sixteen warps in two pairs of 4-warp groups.  Tiles alternate between the pairs (tile
+// counter parity); within a pair the two groups split the accumulator's columns in halves.
+//   pass 1: thread `s` of a group owns stacked row s over its 64 key columns; at the end of the run the
+//           four groups' (shift, sum) pairs meet in shared memory and one group publishes the row's
+//           partial with one 8-byte store.
+//   pass 2: thread `jl` owns key j0 + jl over its half of the stacked rows; the second group of the pair
+//           hands its partial sum over through shared memory, the first adds the two and stores.
+__device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int pair, int half) {
+  Barriers* bars = &sh->bars;
+  const int s = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
+  const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
+  int tc = 0, p1c = 0;
+  bool gone = false;   // a wait ran out: keep only the barriers
+  for_each_segment(a, [&](int pass, int run) {
+    const Run rn = run_info(a, run);
+    const UnitInfo u = unit_info(a, rn.unit);
+    if (pass == 0) {
+      const int i = obs_row(a, u, s);
+      const float c = sh->c[i < a.r ? i : 0];
+      const int last = a.n - a.r + i;                       // last visible key of this row
+      float M = -INFINITY, Z = 0.f;
+      for (int t = 0; t < rn.cnt; ++t, ++tc) {
+        if ((tc & 1) != pair || gone) continue;
+        const int acc = pair * 2 + ((tc >> 1) & 1), aph = (tc >> 2) & 1;
+        if (!mbar_wait(&bars->acc_full[acc], aph, a.status)) { gone = true; continue; }
+        tc_fence_after();
+        const int j0 = (rn.blk0 + t) * kKeyTile + 64 * half;
+        const bool full = (rn.blk0 + t) * kKeyTile + kKeyTile - 1 <= a.n - a.r;   // no key of the tile is masked
+        const uint32_t taddr = lane_base + (uint32_t)(acc * 128 + 64 * half);
+        uint32_t ra[32];
+        // One chunk at a time: load, wait, fold.  The other warps of the scheduler fill the load latency;
+        // keeping a second load in flight costs registers and ties the exponentials to its completion.
+        tmem_ld32_issue(taddr, ra);
+        tmem_ld_wait(ra);
+        fold_chunk(ra, full, j0, last, c, M, Z);
+        tmem_ld32_issue(taddr + 32, ra);
+        tmem_ld_wait(ra);
+        tc_fence_before();
+        mbar_arrive(&bars->acc_empty[acc]);                  // the accumulator is free for the next product
+        fold_chunk(ra, full, j0 + 32, last, c, M, Z);
+      }
+      // All sixteen warps meet here once per run, also after a wait has run out, so that nobody is left
+      // at the barrier.  Two slots: the others can be at most one run ahead of the publishing group's read.
+      const int slot = p1c & 1, who = pair * 2 + half;
+      ++p1c;
+      if (who != 0) sh->p1_part[slot][who - 1][s] = make_float2(M, Z);
+      group_sync(5, 512);
+      if (who == 0 && !gone) {
+        float m = M;
+#pragma unroll
+        for (int w = 0; w < 3; ++w) m = fmaxf(m, sh->p1_part[slot][w][s].x);
+        float z = Z > 0.f ? Z * fast_exp2(M - m) : 0.f;
+#pragma unroll
+        for (int w = 0; w < 3; ++w) {
+          const float2 e = sh->p1_part[slot][w][s];
+          if (e.y > 0.f) z += e.y * fast_exp2(e.x - m);
+        }
+        st_partial(&a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s], make_float2(m, z));
+      }
+    } else {
+      const int jl = s;
+      const int split = ((u.npad / 16 + 1) / 2) * 16;
+      const int c_lo = half ? split : 0, c_hi = half ? u.npad : split;   // this group's accumulator columns
+      const bool fast = a.r <= 128 && u.rows == 128;
+      const float* cs = sh->cs2[u.rb & 1];
+      for (int t = 0; t < rn.cnt; ++t, ++tc) {
+        if ((tc & 1) != pair) continue;
+        const int buf = (tc >> 1) & 1, acc = pair * 2 + buf, aph = (tc >> 2) & 1;
+        const int j0 = (rn.blk0 + t) * kKeyTile, j = j0 + jl;
+        float sum = 0.f;
+        if (!gone && !mbar_wait(&bars->acc_full[acc], aph, a.status)) gone = true;
+        if (!gone) {
+          tc_fence_after();
+          const bool full = j0 + kKeyTile - 1 <= a.n - a.r;
+          const uint32_t taddr = lane_base + (uint32_t)(acc * 128);
+          if (full && fast) {
+            sum = half ? column_sum_fast<1>(a, taddr) : column_sum_fast<0>(a, taddr);
+          } else {
+            // The product wrote exactly npad (a multiple of 16) columns; those past `rows` belong to no row.
+#pragma unroll 1
+            for (int s0 = c_lo; s0 < c_hi; s0 += 16) {
+              uint32_t v[16];
+              tmem_ld16_issue(taddr + s0, v);
+              tmem_ld_wait16(v);
+#pragma unroll
+              for (int t2 = 0; t2 < 16; ++t2) {
+                const int sr = s0 + t2;
+                const bool vis = sr < u.rows && (full || j <= a.n - a.r + obs_row(a, u, sr));
+                if (vis) sum += fast_exp2(__uint_as_float(v[t2]) * cs[sr]);
+              }
+            }
+          }
+          tc_fence_before();
+          mbar_arrive(&bars->acc_empty[acc]);
+        }
+        // The two groups of the pair meet here once per tile, also after a wait has run out.  Two slots:
+        // the second group can be at most one tile ahead of the first group's read.
+        if (half == 1) sh->p2_part[pair][buf][jl] = sum;
+        group_sync(6 + pair, 256);
+        if (half == 0 && !gone && j < a.n) a.s_raw[(size_t)rn.unit * a.n + j] = sum + sh->p2_part[pair][buf][jl];
+      }
+    }
+  });
+}
+
+// nu of the 64 value rows of one V-ring stage: two adjacent lanes share a row (one half of its 16-byte
+// chunks each, in an order that keeps them on different banks), square and add in FP32, and meet by shuffle.
+template <typename T>
+__device__ __forceinline__ float half_row_sq(const char* stage, int row, int sub, int D) {
+  float acc = 0.f;
+  if (D == 128) {
+    const char* base = stage + sub * kVSubBytes + row * 128;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const uint4 q = *reinterpret_cast<const uint4*>(base + (((c ^ sub) ^ (row & 7)) << 4));
+      float f[8];
+      Vec16<T>::widen(q, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+    }
+  } else {
+    const char* base = stage + row * 128;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint4 q = *reinterpret_cast<const uint4*>(base + (((sub * 4 + c) ^ (row & 7)) << 4));
+      float f[8];
+      Vec16<T>::widen(q, f);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+    }
+  }
+  return acc;
+}
+
+// Merge / value-norm group (four warps).  Per step of the fixed sequence:
+//  1. the value rows that go with the step's pass-1 run, as they arrive in the V ring: nu_j = |V_j|^2;
+//  2. for the run whose pass 2 comes one step later: thread `s` waits until the partials of row s have
+//     arrived from all runs of the row block, merges them in run order into the row's offset and writes
+//     the row's offset extension into shared memory for the MMA.
+__device__ void aux_group(const TcArgs& a, Shared* sh, char* tiles) {
   Barriers* bars = &sh->bars;
   const int s = threadIdx.x & 127;
-  int prev_unit = -1, uc = 0;
+  const int G = (int)gridDim.x, first = (int)blockIdx.x;
+  const int nr = (a.n_runs - first + G - 1) / G;
+  int vc = 0, mc = 0;
   bool dead = false;   // a wait ran out: nothing more is delivered (the MMA warp's own waits then run out too)
-  for (int run = blockIdx.x; run < a.n_runs && !dead; run += gridDim.x) {
-    const Run rn = run_info(a, run);
-    if (rn.unit == prev_unit) continue;
-    prev_unit = rn.unit;
+  for (int k = 0; k < nr + a.lead - 1 && !dead; ++k) {
+    if (k < nr && a.prior) {
+      const Run rn = run_info(a, first + k * G);
+      const UnitInfo u = unit_info(a, rn.unit);
+      if (u.rb == 0) {
+        const int row = s >> 1, sub = s & 1;
+        for (int t = 0; t < 2 * rn.cnt && !dead; ++t, ++vc) {
+          const int vs = vc & 1;
+          if (!mbar_wait(&bars->v_full[vs], (vc >> 1) & 1, a.status)) { dead = true; break; }
+          const char* stage = tiles + kOffV + vs * kVStageBytes;
+          float sq = a.bf16 ? half_row_sq<__nv_bfloat16>(stage, row, sub, a.D) : half_row_sq<__half>(stage, row, sub, a.D);
+          sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+          mbar_arrive(&bars->v_empty[vs]);
+          const int j = rn.blk0 * kKeyTile + t * kVRows + row;
+          if (sub == 0 && j < a.n) a.nu[(size_t)u.bh * a.n + j] = sq;
+        }
+      }
+    }
+    const int jm = k - a.lead + 1;
+    if (jm < 0 || jm >= nr || dead) continue;
+    const Run rn = run_info(a, first + jm * G);
     const UnitInfo u = unit_info(a, rn.unit);
-    const int slot = uc & 1;
-    if (!mbar_wait(&bars->ext_empty[slot], ((uc >> 1) & 1) ^ 1, a.status)) break;
-    ++uc;
+    const int slot = mc & 1;
+    if (!mbar_wait(&bars->ext_empty[slot], ((mc >> 1) & 1) ^ 1, a.status)) break;
+    ++mc;
     const float2* p = a.partial + (size_t)rn.unit * a.rpu * 128 + s;
     float Mx = -INFINITY, Zs = 0.f;
     for (int t0 = 0; t0 < a.rpu && !dead; t0 += 16) {     // 16 loads in flight per thread
@@ -571,7 +760,7 @@ __device__ void merge_group(const TcArgs& a, Shared* sh, char* ext_smem) {
         w1 = (uint32_t)__half_as_ushort(h3);
       }
     }
-    uint4* row = reinterpret_cast<uint4*>(ext_smem + slot * kExtBytes + s * 32);
+    uint4* row = reinterpret_cast<uint4*>(tiles + kOffExt + slot * kExtBytes + s * 32);
     row[0] = make_uint4(w0, w1, 0u, 0u);
     row[1] = make_uint4(w0, w1, 0u, 0u);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads it through the async proxy
@@ -579,97 +768,11 @@ __device__ void merge_group(const TcArgs& a, Shared* sh, char* ext_smem) {
   }
 }
 
-// Sixty-four stacked rows of a key's column, rows [64 HALF, 64 HALF + 64): adds 2^{c D} of each.  The
-// column indices are compile-time constants, so every c comes straight from the kernel's parameter
-// bank as an operand of the multiply.
-template <int HALF>
-__device__ __forceinline__ float column_sum_fast(const TcArgs& a, uint32_t taddr) {
-  float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    uint32_t r[16];
-    tmem_ld16_issue(taddr + 64 * HALF + 16 * q, r);
-    tmem_ld_wait16(r);
-#pragma unroll
-    for (int t = 0; t < 16; t += 4) {
-      z0 += fast_exp2(__uint_as_float(r[t]) * a.cs[64 * HALF + 16 * q + t]);
-      z1 += fast_exp2(__uint_as_float(r[t + 1]) * a.cs[64 * HALF + 16 * q + t + 1]);
-      z2 += fast_exp2(__uint_as_float(r[t + 2]) * a.cs[64 * HALF + 16 * q + t + 2]);
-      z3 += fast_exp2(__uint_as_float(r[t + 3]) * a.cs[64 * HALF + 16 * q + t + 3]);
-    }
-  }
-  return (z0 + z1) + (z2 + z3);
-}
-
-// Pass-2 softmax groups: two groups of four warps share each accumulator; thread `jl` of either group owns
-// key j0 + jl, group 0 over the first half of the stacked rows (accumulator columns), group 1 over the
-// rest.  Group 1 hands its partial sum over through shared memory; group 0 adds the two and stores.
-__device__ __forceinline__ void column_sum_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int half) {
-  Barriers* bars = &sh->bars;
-  const int jl = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
-  int it = 0, prev_unit = -1;
-  bool gone = false;     // an accumulator wait ran out: keep only the group barrier
-  UnitInfo u = unit_info(a, 0);
-  int c_lo = 0, c_hi = 0;   // this group's accumulator columns
-  bool fast = false;
-  for (int run = blockIdx.x; run < a.n_runs; run += gridDim.x) {
-    const Run rn = run_info(a, run);
-    if (rn.unit != prev_unit) {
-      prev_unit = rn.unit;
-      u = unit_info(a, rn.unit);
-      const int split = ((u.npad / 16 + 1) / 2) * 16;
-      c_lo = half ? split : 0;
-      c_hi = half ? u.npad : split;
-      fast = a.r <= 128 && u.rows == 128;
-    }
-    const float* cs = sh->cs2[u.rb & 1];
-    for (int t = 0; t < rn.cnt; ++t, ++it) {
-      const int acc = it & 1, aph = (it >> 1) & 1;
-      const int j0 = (rn.blk0 + t) * kKeyTile, j = j0 + jl;
-      float sum = 0.f;
-      if (!gone && !mbar_wait(&bars->acc_full[1][acc], aph, a.status)) gone = true;
-      if (!gone) {
-        tc_fence_after();
-        const bool full = j0 + kKeyTile - 1 <= a.n - a.r;
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((2 + acc) * 128);
-        if (full && fast) {
-          sum = half ? column_sum_fast<1>(a, taddr) : column_sum_fast<0>(a, taddr);
-        } else {
-          // The product wrote exactly npad (a multiple of 16) columns; those past `rows` belong to no row.
-#pragma unroll 1
-          for (int s0 = c_lo; s0 < c_hi; s0 += 16) {
-            uint32_t v[16];
-            tmem_ld16_issue(taddr + s0, v);
-            tmem_ld_wait16(v);
-#pragma unroll
-            for (int t2 = 0; t2 < 16; ++t2) {
-              const int sr = s0 + t2;
-              const bool vis = sr < u.rows && (full || j <= a.n - a.r + obs_row(a, u, sr));
-              if (vis) sum += fast_exp2(__uint_as_float(v[t2]) * cs[sr]);
-            }
-          }
-        }
-        tc_fence_before();
-        mbar_arrive(&bars->acc_empty[1][acc]);
-      }
-      // Both groups meet here once per tile, also after a wait has run out, so that nobody is left at
-      // the barrier.  Two slots: group 1 can be at most one tile ahead of group 0's read.
-      if (half == 1) sh->p2_part[it & 1][jl] = sum;
-      group_sync(4, 256);
-      if (half == 0 && !gone && j < a.n) a.s_raw[(size_t)rn.unit * a.n + j] = sum + sh->p2_part[it & 1][jl];
-    }
-  }
-}
-
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
-                const __grid_constant__ TcArgs a) {
+                const __grid_constant__ CUtensorMap vmap, const __grid_constant__ TcArgs a) {
   extern __shared__ char smem_raw[];
   char* tiles = reinterpret_cast<char*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  char* q_smem[2] = {tiles, tiles + kQBytes + kKRingBytes};
-  char* k_ring[2] = {tiles + kQBytes, tiles + 2 * kQBytes + kKRingBytes};
-  char* ext_smem = tiles + 2 * (kQBytes + kKRingBytes);   // pass 2: two offset extensions (current, next)
-  char* fold_smem = ext_smem + 2 * kExtBytes;             // pass 2: the constant tile
   Shared* sh = reinterpret_cast<Shared*>(tiles + kSmemTiles);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -683,32 +786,34 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     // three parts of a row's extension twice, once per 16-byte half of the row
     const uint32_t one = a.bf16 ? (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(kFold))
                                 : (uint32_t)__half_as_ushort(__float2half_rn(kFold));
-    uint4* f = reinterpret_cast<uint4*>(fold_smem);
+    uint4* f = reinterpret_cast<uint4*>(tiles + kOffExt + 2 * kExtBytes);
     for (int t = threadIdx.x; t < kExtBytes / 16; t += kThreads) f[t] = make_uint4(one | (one << 16), one, 0u, 0u);
   }
   // Q rows a TMA box never covers (row blocks with fewer than 128 rows) must read as zeros, not as
   // whatever the last kernel left: zero both Q buffers once, before any bulk copy is issued.
-  for (int p = 0; p < 2; ++p) {
-    uint4* z = reinterpret_cast<uint4*>(q_smem[p]);
-    for (int t = threadIdx.x; t < kQBytes / 16; t += kThreads) z[t] = make_uint4(0, 0, 0, 0);
+  {
+    uint4* z = reinterpret_cast<uint4*>(tiles + kOffQ);
+    for (int t = threadIdx.x; t < 2 * kQBytes / 16; t += kThreads) z[t] = make_uint4(0, 0, 0, 0);
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   if (threadIdx.x == 0) {
     Barriers* bars = &sh->bars;
     for (int p = 0; p < 2; ++p) {
       mbar_init(&bars->q_full[p], 1);
-      for (int s = 0; s < kStages; ++s) {
-        mbar_init(&bars->k_full[p][s], 1);
-        mbar_init(&bars->k_empty[p][s], 1);
-      }
-      for (int s = 0; s < 2; ++s) {
-        mbar_init(&bars->acc_full[p][s], 1);
-        mbar_init(&bars->acc_empty[p][s], 256);
-      }
+      mbar_init(&bars->q_empty[p], 1);
+      mbar_init(&bars->v_full[p], 1);
+      mbar_init(&bars->v_empty[p], 128);
       mbar_init(&bars->ext_full[p], 128);
       mbar_init(&bars->ext_empty[p], 1);
     }
-    sh->p2_unit = 0;
+    for (int s = 0; s < kKStages; ++s) {
+      mbar_init(&bars->k_full[s], 1);
+      mbar_init(&bars->k_empty[s], 1);
+    }
+    for (int s = 0; s < 4; ++s) {
+      mbar_init(&bars->acc_full[s], 1);
+      mbar_init(&bars->acc_empty[s], 256);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // all 512 TMEM columns: four 128-column accumulators
@@ -721,19 +826,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   const uint32_t tmem_base = sh->tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) producer(a, &qmap, &kmap, sh, 0, q_smem[0], k_ring[0]);
+    if (lane == 0) producer(a, &qmap, &kmap, sh, tiles);
   } else if (warp == 1) {
-    if (lane == 0) mma_issuer(a, sh, 0, q_smem[0], k_ring[0], ext_smem, fold_smem, tmem_base);
+    if (lane == 0) mma_issuer(a, sh, tiles, tmem_base);
   } else if (warp == 2) {
-    if (lane == 0) producer(a, &qmap, &kmap, sh, 1, q_smem[1], k_ring[1]);
+    if (lane == 0 && a.prior) v_producer(a, &vmap, sh, tiles);
   } else if (warp == 3) {
-    if (lane == 0) mma_issuer(a, sh, 1, q_smem[1], k_ring[1], ext_smem, fold_smem, tmem_base);
-  } else if (warp < 12) {
-    row_stats_group(a, sh, tmem_base, (warp - 4) >> 2);
+    // idle
   } else if (warp < 20) {
-    column_sum_group(a, sh, tmem_base, (warp - 12) >> 2);
+    softmax_group(a, sh, tmem_base, (warp - 4) >> 3, ((warp - 4) >> 2) & 1);
   } else {
-    merge_group(a, sh, ext_smem);
+    aux_group(a, sh, tiles);
   }
 
   tc_fence_before();
@@ -779,8 +882,8 @@ bool make_map(CUtensorMap* m, const void* base, int bf16, int d, long long token
 
 bool score_tc_available() { return encode_fn() != nullptr; }
 
-ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float* s_raw, float2* partial,
-                             int* status, cudaStream_t st) {
+ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
+                             float2* partial, int* status, cudaStream_t st) {
   static int n_sm = 0;
   static bool configured = false;
   if (!configured) {
@@ -797,30 +900,42 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, float
   a.n_blk = pl.n_blk; a.D = pl.d;
   const long long tiles = (long long)units * pl.n_blk;
   const long long ch = tiles / ((long long)n_sm * 8);
-  a.CH = ch < 1 ? 1 : (ch > 8 ? 8 : (int)ch);
+  a.CH = ch < 1 ? 1 : (ch > 4 ? 4 : (int)ch);
   a.rpu = (pl.n_blk + a.CH - 1) / a.CH;
   a.n_runs = units * a.rpu;
-  // keep about 48 MiB of keys between the two passes, which L2 still holds next to the rest of the traffic
-  const long long unit_bytes = (long long)pl.n * pl.d * pl.es;
-  const long long lag = (48LL << 20) / (unit_bytes * pl.n_rb > 0 ? unit_bytes : 1) * pl.n_rb;
-  a.lag = lag < 2 * pl.n_rb ? 2 * pl.n_rb : (lag > 4096 ? 4096 : (int)lag);
+  const int grid = a.n_runs < n_sm ? a.n_runs : n_sm;
+  // Pass 2 of a run follows its pass 1 by `lead` steps.  At least as many as the steps a row block's runs
+  // are spread over, so that a wait only depends on earlier work; beyond that, as many as keep about
+  // 40 MB of keys between the passes (L2 still holds that next to the rest of the traffic).
+  const long long step_bytes = (long long)grid * a.CH * kKeyTile * pl.d * pl.es;
+  long long lead = (40LL << 20) / (step_bytes > 0 ? step_bytes : 1);
+  if (lead > 3) lead = 3;
+  const long long spread = (a.rpu - 1 + grid - 1) / grid;
+  if (lead < spread) lead = spread;
+  if (lead < 1) lead = 1;
+  a.lead = (int)lead;
   a.bf16 = pl.dtype == AHAKV_BF16;
+  a.prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0 && v != nullptr && nu != nullptr;
   a.log2G = log2f((float)pl.G);
   for (int i = 0; i < kMaxRows; ++i) a.c[i] = pl.rows.c[i];
   for (int t = 0; t < 128; ++t) a.cs[t] = pl.r <= 128 ? pl.rows.c[t % pl.r] : 0.f;
-  a.partial = partial; a.s_raw = s_raw;
+  a.partial = partial; a.s_raw = s_raw; a.nu = nu;
   a.status = status;
 
-  CUtensorMap qmap, kmap;
+  CUtensorMap qmap, kmap, vmap;
   const int q_box_rows = pl.r <= 128 ? pl.r : 128, q_box_heads = pl.r <= 128 ? pl.heads_per_rb : 1;
   if (!make_map(&qmap, q, a.bf16, pl.d, pl.r, pl.Hq, pl.B, pl.qs, pl.es, q_box_rows, q_box_heads) ||
       !make_map(&kmap, k, a.bf16, pl.d, pl.n, pl.Hkv, pl.B, pl.ks, pl.es, kKeyTile, 1))
     return AHAKV_ERR_CUDA;
+  if (a.prior) {
+    if (!make_map(&vmap, v, a.bf16, pl.d, pl.n, pl.Hkv, pl.B, pl.vs, pl.es, kVRows, 1)) return AHAKV_ERR_CUDA;
+  } else {
+    vmap = kmap;   // never used
+  }
 
   // every partial starts as NaN: "not published yet"
   if (cudaMemsetAsync(partial, 0xff, (size_t)a.n_runs * 128 * sizeof(float2), st) != cudaSuccess) return AHAKV_ERR_CUDA;
-  const int grid = a.n_runs < n_sm ? a.n_runs : n_sm;
-  void* args[] = {&qmap, &kmap, &a};
+  void* args[] = {&qmap, &kmap, &vmap, &a};
   const cudaError_t e = cudaLaunchCooperativeKernel((const void*)score_tc_kernel, dim3(grid), dim3(kThreads), args,
                                                     (size_t)kSmemBytes, st);
   count_launch();
