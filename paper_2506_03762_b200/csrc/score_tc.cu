@@ -209,15 +209,6 @@ __device__ __forceinline__ uint32_t umma_idesc(int M, int N, int bf16) {
   return d;
 }
 
-__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, int accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
 // 32 consecutive FP32 columns of this thread's TMEM lane: issue now, use after tmem_ld_wait(r).
 __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r) {
   asm volatile(
@@ -404,17 +395,31 @@ __device__ void v_producer(const TcArgs& a, const CUtensorMap* vmap, Shared* sh,
   }
 }
 
-// MMA issuer.  Pass 1: D[rows x keys] = Q K^T.  Pass 2: D[keys x rows] = K Q^T - off / c.
+// One k-step of a product.  The descriptors differ from their tile's base only in the address field
+// (bits 0-13, in 16-byte units), so a k-step costs one add per operand.
+template <int ACC>
+__device__ __forceinline__ void umma_step(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
+  const uint32_t accumulate = ACC;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// MMA issuer (one thread).
+// Pass 1: D[rows x keys] = Q K^T.  Pass 2: D[keys x rows] = K Q^T - off / c.
 __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tmem_base) {
   Barriers* bars = &sh->bars;
   int tc = 0, sc = 0, pc = 0;
   bool ok = true;
   const uint64_t fold_desc = umma_desc_ext(smem_u32(tiles + kOffExt + 2 * kExtBytes));
+  const int nk = a.D / 16;
   for_each_segment(a, [&](int pass, int run) {
     if (!ok) return;
     const Run rn = run_info(a, run);
     const int qb = sc & 1;
-    char* q_smem = tiles + kOffQ + qb * kQBytes;
     if (!(ok = mbar_wait(&bars->q_full[qb], (sc >> 1) & 1, a.status))) return;
     uint32_t idesc = umma_idesc(128, 128, a.bf16);
     uint64_t ext_desc = 0;
@@ -433,16 +438,19 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tm
       if (!(ok = mbar_wait(&bars->k_full[stage], ph, a.status))) return;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 128);
-      char* k_smem = tiles + kOffK + stage * kKStageBytes;
-      for (int kk = 0; kk < a.D / 16; ++kk) {
-        const int sub = kk >> 2, koff = (kk & 3) * 32;
-        const uint64_t qd = umma_desc(smem_u32(q_smem + sub * kSubTileBytes) + koff);
-        const uint64_t kd = umma_desc(smem_u32(k_smem + sub * kSubTileBytes) + koff);
-        if (pass == 0) umma(d_tmem, qd, kd, idesc, kk > 0);
-        else umma(d_tmem, kd, qd, idesc, kk > 0);
+      const uint32_t q_addr = smem_u32(tiles + kOffQ + qb * kQBytes), k_addr = smem_u32(tiles + kOffK + stage * kKStageBytes);
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        // k-step kk reads 32 bytes at offset (kk & 3) * 32 of sub-tile kk >> 2
+        const uint32_t off = (uint32_t)((kk >> 2) * kSubTileBytes + (kk & 3) * 32);
+        const uint64_t qd = umma_desc(q_addr + off), kd = umma_desc(k_addr + off);
+        if (kk < nk) {
+          if (kk == 0) umma_step<0>(d_tmem, pass == 0 ? qd : kd, pass == 0 ? kd : qd, idesc);
+          else umma_step<1>(d_tmem, pass == 0 ? qd : kd, pass == 0 ? kd : qd, idesc);
+        }
       }
       // pass 2: D -= off / c, as one more k-step over the constant tile and the rows' offset extensions
-      if (pass == 1) umma(d_tmem, fold_desc, ext_desc, idesc, 1);
+      if (pass == 1) umma_step<1>(d_tmem, fold_desc, ext_desc, idesc);
       tc_commit(&bars->k_empty[stage]);
       tc_commit(&bars->acc_full[acc]);
     }
