@@ -7,9 +7,9 @@
 // A normalised column sum needs each row's softmax statistics over ALL keys
 // first, so every tile is visited twice:
 //
-//   pass 1 (rows on TMEM lanes):  D = Q . K^T   -> per-row (shift, sum of 2^{c w - shift})
-//                                 of a run of tiles, stored to global memory as one
-//                                 8-byte partial per row and run.
+//   pass 1 (rows on TMEM lanes):  D = Q . K^T   -> per-row log2 sum of 2^{c w} over a run of
+//                                 tiles, stored to global memory as one 4-byte partial
+//                                 per row and run.
 //   pass 2 (keys on TMEM lanes):  D = K . Q^T - off/c -> each thread owns one key and adds
 //                                 2^{c D} over the rows: the column sum needs no
 //                                 cross-thread traffic and no per-row constant but c.
@@ -29,10 +29,10 @@
 //
 // Between the passes there are no flags, counters or fences.  The partials start
 // as NaN (the host clears them before the launch) and each is published by a single
-// 8-byte store, so a reader knows a partial is there when it no longer reads NaN.
+// 4-byte store, so a reader knows a partial is there when it no longer reads NaN.
 // Every CTA merges, for the run its pass 2 turns to next, the partials of all
-// runs of that row block into one offset per row by itself (a 4-warp group does this
-// one step ahead of the MMAs, off the critical path), always in run order: the
+// runs of that row block into one offset per row by itself (two warps do this up to
+// two runs ahead of the MMAs, off the critical path), always in run order: the
 // result does not depend on who finished first.
 //
 // The row offsets ride in the product itself: the merged offset of a row becomes
@@ -45,8 +45,8 @@
 // the 32-byte swizzle orders them.
 //
 // The value rows of the keys of each pass-1 tile stream through a small ring of their
-// own (a second TMA warp, evict-first in L2) and the same 4-warp group squares and
-// adds them: nu_j = |V_j|^2 costs no launch and no second sweep of HBM.
+// own (evict-first in L2); four warps square and add them: nu_j = |V_j|^2 costs no
+// launch and no second sweep of HBM.
 //
 // The kernel is launched cooperatively with at most one CTA per SM, which guarantees
 // that the CTAs a partial comes from are running; a wait only ever depends on work
@@ -63,8 +63,9 @@ namespace {
 constexpr int kKStages = 3;                // K-tile ring depth
 constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 16-bit elements, 128-byte swizzled
 constexpr int kVRows = 64;                 // value rows per V-ring stage
+constexpr int kVStages = 2;
 constexpr int kVSubBytes = kVRows * 128;
-constexpr int kThreads = 768;              // 4 service warps, 16 softmax warps, the 4-warp merge / value-norm group
+constexpr int kThreads = 768;              // TMA warp, MMA warp, 2 merge warps, 16 softmax warps, 4 value-norm warps
 constexpr long long kWaitLimitNs = 1000000000LL;   // 1 s
 constexpr float kFold = 256.f;             // value of the constant tile; offsets are stored divided by it
 
@@ -79,7 +80,7 @@ struct TcArgs {
   float log2G;
   float c[kMaxRows];     // lambda_i log2(e) per observation row
   float cs[128];         // the same per stacked row of a row block (r <= 128 only)
-  float2* partial;   // [unit][run][128]
+  float* partial;    // [unit][run][128]: log2 of a row's sum of 2^{c w} over the run's keys
   float* s_raw;      // [unit][n]
   float* nu;         // [B * Hkv][n]
   int* status;
@@ -89,7 +90,7 @@ struct TcArgs {
 struct __align__(8) Barriers {
   unsigned long long q_full[2], q_empty[2];
   unsigned long long k_full[kKStages], k_empty[kKStages];
-  unsigned long long v_full[2], v_empty[2];
+  unsigned long long v_full[kVStages], v_empty[kVStages];
   unsigned long long acc_full[4], acc_empty[4];
   unsigned long long ext_full[2], ext_empty[2];   // offset extension of a run's row block: merge group -> MMA
 };
@@ -100,6 +101,7 @@ struct Shared {
   int pad_;
   float c[kMaxRows];            // lambda_i * log2(e) per observation row
   float cs2[2][128];            // c per stacked row, by row block parity (r > 128 has two kinds of block)
+  int vis_off[2][128];          // per stacked row: n - r + its observation row = the last key it may see
   float2 p1_part[2][3][128];    // pass 1: statistics of the three groups that do not publish
   float p2_part[2][2][128];     // pass 2: partial column sums of the second half of the rows, per pair
 };
@@ -111,7 +113,7 @@ constexpr int kExtBytes = 128 * 32;                      // 128 rows x 16 16-bit
 constexpr int kOffQ = 0;
 constexpr int kOffK = kOffQ + 2 * kQBytes;
 constexpr int kOffV = kOffK + kKStages * kKStageBytes;
-constexpr int kOffExt = kOffV + 2 * kVStageBytes;        // two extensions, then the constant tile
+constexpr int kOffExt = kOffV + kVStages * kVStageBytes;        // two extensions, then the constant tile
 constexpr int kSmemTiles = kOffExt + 3 * kExtBytes;      // 204 KiB
 constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 12288 /*barriers, constants, exchange*/;
 static_assert(sizeof(Shared) <= 12288, "Shared outgrew its reservation");
@@ -257,13 +259,13 @@ __device__ __forceinline__ void group_sync(int id, int threads) {
 }
 
 // One partial, straight from L2 (other CTAs write it while this one polls).
-__device__ __forceinline__ float2 ld_partial(const float2* p) {
+__device__ __forceinline__ float2 ld_partial2(const float2* p) {   // two adjacent rows
   float2 v;
   asm volatile("ld.relaxed.gpu.global.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_partial(float2* p, float2 v) {
-  asm volatile("st.relaxed.gpu.global.v2.f32 [%0], {%1, %2};" ::"l"(p), "f"(v.x), "f"(v.y) : "memory");
+__device__ __forceinline__ void st_partial(float* p, float v) {
+  asm volatile("st.relaxed.gpu.global.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
 }
 
 // ---- work decomposition ----------------------------------------------------------------------------------
@@ -326,72 +328,174 @@ __device__ __forceinline__ void for_each_segment(const TcArgs& a, F f) {
   }
 }
 
+// The fixed sequence again, as a cursor that can be advanced one segment at a time.
+struct SegCursor {
+  int k, sub;
+};
+__device__ __forceinline__ bool seg_next(const TcArgs& a, int nr, SegCursor& c, int& pass, int& run) {
+  const int G = (int)gridDim.x, first = (int)blockIdx.x;
+  while (c.k < nr + a.lead) {
+    if (c.sub == 0) {
+      c.sub = 1;
+      if (c.k < nr) { pass = 0; run = first + c.k * G; return true; }
+    }
+    c.sub = 0;
+    const int k = c.k++;
+    if (k >= a.lead) { pass = 1; run = first + (k - a.lead) * G; return true; }
+  }
+  return false;
+}
+
+// The next 64 value rows to fetch or to square: stage t of the run at step k (first row block of a KV
+// head only).
+struct VCursor {
+  int k, t, cnt, row0, b, h, bh;
+};
+__device__ __forceinline__ bool v_seek(const TcArgs& a, int nr, VCursor& c) {
+  const int G = (int)gridDim.x, first = (int)blockIdx.x;
+  for (; c.k < nr; ++c.k) {
+    const Run rn = run_info(a, first + c.k * G);
+    const UnitInfo u = unit_info(a, rn.unit);
+    if (u.rb != 0) continue;
+    c.t = 0; c.cnt = 2 * rn.cnt; c.row0 = rn.blk0 * kKeyTile; c.b = u.b; c.h = u.h; c.bh = u.bh;
+    return true;
+  }
+  return false;
+}
+__device__ __forceinline__ bool v_advance(const TcArgs& a, int nr, VCursor& c) {
+  if (++c.t < c.cnt) return true;
+  ++c.k;
+  return v_seek(a, nr, c);
+}
+
 // ---- roles --------------------------------------------------------------------------------------------
-// TMA producer of Q and K tiles.
-__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, Shared* sh, char* tiles) {
+// TMA producer: one thread feeds two independent streams, whichever has a free slot: Q and K tiles in
+// the order of the fixed sequence, and the value rows that go with the pass-1 key tiles.
+__device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, const CUtensorMap* vmap,
+                         Shared* sh, char* tiles) {
   Barriers* bars = &sh->bars;
   const int n_sub = a.D / 64;
   const int q_rows = a.r <= 128 ? a.hb * a.r : 128;
   const int q_bytes = n_sub * q_rows * 128, k_bytes = n_sub * kSubTileBytes;
   const unsigned long long once = policy_evict_first();
-  int tc = 0, sc = 0;
-  bool ok = true;
-  for_each_segment(a, [&](int pass, int run) {
-    if (!ok) return;
-    const Run rn = run_info(a, run);
-    const UnitInfo u = unit_info(a, rn.unit);
-    const int qb = sc & 1;
-    char* q_smem = tiles + kOffQ + qb * kQBytes;
-    if (!(ok = mbar_wait(&bars->q_empty[qb], ((sc >> 1) & 1) ^ 1, a.status))) return;
-    mbar_expect_tx(&bars->q_full[qb], q_bytes);
-    for (int s = 0; s < n_sub; ++s) {
-      if (a.r <= 128) tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, 0, u.h * a.G + u.rb * a.hb, u.b);
-      else tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, u.rb * 128, u.h, u.b);
-    }
-    ++sc;
-    for (int t = 0; t < rn.cnt; ++t, ++tc) {
-      const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
-      if (!(ok = mbar_wait(&bars->k_empty[stage], ph ^ 1, a.status))) return;
-      mbar_expect_tx(&bars->k_full[stage], k_bytes);
-      char* dst = tiles + kOffK + stage * kKStageBytes;
-      for (int s = 0; s < n_sub; ++s) {
-        // the second read of a key tile is its last: let L2 drop it first
-        if (pass == 0) tma_load_4d(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b);
-        else tma_load_4d_hint(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b, once);
+  const int G = (int)gridDim.x, first = (int)blockIdx.x;
+  const int nr = (a.n_runs - first + G - 1) / G;
+
+  // K stream state
+  SegCursor sc_cur = {0, 0};
+  int pass = 0, run = 0, tc = 0, sc = 0, t = 0;
+  Run rn = run_info(a, first);
+  UnitInfo u = unit_info(a, rn.unit);
+  bool k_live = seg_next(a, nr, sc_cur, pass, run), q_due = true;
+  if (k_live) { rn = run_info(a, run); u = unit_info(a, rn.unit); }
+  // V stream state
+  VCursor vcur;
+  vcur.k = 0;
+  bool v_live = a.prior && v_seek(a, nr, vcur);
+  int vc = 0;
+
+  long long idle_since = -1;
+  while (k_live || v_live) {
+    bool progress = false;
+    if (k_live) {
+      if (q_due) {
+        const int qb = sc & 1;
+        if (mbar_try(&bars->q_empty[qb], ((sc >> 1) & 1) ^ 1)) {
+          char* q_smem = tiles + kOffQ + qb * kQBytes;
+          mbar_expect_tx(&bars->q_full[qb], q_bytes);
+          for (int s = 0; s < n_sub; ++s) {
+            if (a.r <= 128) tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, 0, u.h * a.G + u.rb * a.hb, u.b);
+            else tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, u.rb * 128, u.h, u.b);
+          }
+          ++sc;
+          q_due = false;
+          progress = true;
+        }
+      } else {
+        const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
+        if (mbar_try(&bars->k_empty[stage], ph ^ 1)) {
+          mbar_expect_tx(&bars->k_full[stage], k_bytes);
+          char* dst = tiles + kOffK + stage * kKStageBytes;
+          for (int s = 0; s < n_sub; ++s) {
+            // the second read of a key tile is its last: let L2 drop it first
+            if (pass == 0) tma_load_4d(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b);
+            else tma_load_4d_hint(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b, once);
+          }
+          ++tc;
+          if (++t == rn.cnt) {
+            t = 0;
+            q_due = true;
+            k_live = seg_next(a, nr, sc_cur, pass, run);
+            if (k_live) { rn = run_info(a, run); u = unit_info(a, rn.unit); }
+          }
+          progress = true;
+        }
       }
     }
-  });
-  if (!ok) {
-    // wind down: give copies already in flight a bounded time (1 ms) to land before the CTA exits
-    const long long t0 = now_ns();
-    while (now_ns() - t0 < 1000000) __nanosleep(1000);
+    if (v_live) {
+      const int vs = vc % kVStages;
+      if (mbar_try(&bars->v_empty[vs], ((vc / kVStages) & 1) ^ 1)) {
+        mbar_expect_tx(&bars->v_full[vs], n_sub * kVSubBytes);
+        char* dst = tiles + kOffV + vs * kVStageBytes;
+        for (int s = 0; s < n_sub; ++s)
+          tma_load_4d_hint(dst + s * kVSubBytes, vmap, &bars->v_full[vs], s * 64, vcur.row0 + vcur.t * kVRows, vcur.h, vcur.b, once);
+        ++vc;
+        v_live = v_advance(a, nr, vcur);
+        progress = true;
+      }
+    }
+    if (progress) {
+      idle_since = -1;
+    } else {
+      const long long now = now_ns();
+      if (idle_since < 0) idle_since = now;
+      else if (now - idle_since > kWaitLimitNs) {
+        atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
+        // wind down: give copies already in flight a bounded time (1 ms) to land before the CTA exits
+        while (now_ns() - now < 1000000) __nanosleep(1000);
+        return;
+      }
+    }
   }
 }
 
-// TMA producer of the value rows that go with the key tiles of pass 1 (first row block of a KV head only).
-__device__ void v_producer(const TcArgs& a, const CUtensorMap* vmap, Shared* sh, char* tiles) {
+// Value-norm group (four warps, 128 threads): two adjacent lanes share a row of each 64-row stage of the
+// V ring (one half of its 16-byte chunks each, in an order that keeps them on different banks), square
+// and add in FP32 and meet by shuffle: nu_j = |V_j|^2.
+__device__ void v_group(const TcArgs& a, Shared* sh, char* tiles) {
   Barriers* bars = &sh->bars;
-  const int n_sub = a.D / 64;
-  const unsigned long long once = policy_evict_first();
-  int vc = 0;
-  bool ok = true;
-  for_each_segment(a, [&](int pass, int run) {
-    if (pass != 0 || !ok) return;
-    const Run rn = run_info(a, run);
-    const UnitInfo u = unit_info(a, rn.unit);
-    if (u.rb != 0) return;
-    for (int t = 0; t < 2 * rn.cnt; ++t, ++vc) {
-      const int vs = vc & 1;
-      if (!(ok = mbar_wait(&bars->v_empty[vs], ((vc >> 1) & 1) ^ 1, a.status))) return;
-      mbar_expect_tx(&bars->v_full[vs], n_sub * kVSubBytes);
-      char* dst = tiles + kOffV + vs * kVStageBytes;
-      for (int s = 0; s < n_sub; ++s)
-        tma_load_4d_hint(dst + s * kVSubBytes, vmap, &bars->v_full[vs], s * 64, rn.blk0 * kKeyTile + t * kVRows, u.h, u.b, once);
+  const int row = (threadIdx.x & 127) >> 1, sub = threadIdx.x & 1;
+  const int G = (int)gridDim.x, first = (int)blockIdx.x;
+  const int nr = (a.n_runs - first + G - 1) / G;
+  VCursor cc;
+  cc.k = 0;
+  bool cv = v_seek(a, nr, cc);
+  for (int ci = 0; cv; ++ci) {
+    const int vs = ci % kVStages;
+    if (!mbar_wait(&bars->v_full[vs], (ci / kVStages) & 1, a.status)) return;
+    const char* stage = tiles + kOffV + vs * kVStageBytes;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      // head_dim 128: lane `sub` takes sub-tile `sub`, chunks in the order c ^ sub; head_dim 64: chunks
+      // 4 sub .. 4 sub + 3 of the one sub-tile
+      const int chunk = a.D == 128 ? (c ^ sub) : (4 * sub + c);
+      if (a.D == 128 || c < 4) {
+        const uint4 q = *reinterpret_cast<const uint4*>(stage + (a.D == 128 ? sub * kVSubBytes : 0) + row * 128 +
+                                                        ((chunk ^ (row & 7)) << 4));
+        float f[8];
+        if (a.bf16) Vec16<__nv_bfloat16>::widen(q, f);
+        else Vec16<__half>::widen(q, f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e & 3] = fmaf(f[e], f[e], acc[e & 3]);
+      }
     }
-  });
-  if (!ok) {
-    const long long t0 = now_ns();
-    while (now_ns() - t0 < 1000000) __nanosleep(1000);
+    mbar_arrive(&bars->v_empty[vs]);
+    float sq = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+    const int j = cc.row0 + cc.t * kVRows + row;
+    if (sub == 0 && j < a.n) a.nu[(size_t)cc.bh * a.n + j] = sq;
+    cv = v_advance(a, nr, cc);
   }
 }
 
@@ -543,7 +647,7 @@ __device__ __forceinline__ float column_sum_fast(const TcArgs& a, uint32_t taddr
 // counter parity); within a pair the two groups split the accumulator's columns in halves.
 //   pass 1: thread `s` of a group owns stacked row s over its 64 key columns; at the end of the run the
 //           four groups' (shift, sum) pairs meet in shared memory and one group publishes the row's
-//           partial with one 8-byte store.
+//           partial, log2 of the sum, with one 4-byte store.
 //   pass 2: thread `jl` owns key j0 + jl over its half of the stacked rows; the second group of the pair
 //           hands its partial sum over through shared memory, the first adds the two and stores.
 __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int pair, int half) {
@@ -596,7 +700,9 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
           const float2 e = sh->p1_part[slot][w][s];
           if (e.y > 0.f) z += e.y * fast_exp2(e.x - m);
         }
-        st_partial(&a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s], make_float2(m, z));
+        float L = z > 0.f ? m + log2f(z) : -INFINITY;
+        if (L != L) L = INFINITY;                            // NaN inputs: never publish the 'not yet' pattern
+        st_partial(&a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s], L);
       }
     } else {
       const int jl = s;
@@ -604,6 +710,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
       const int c_lo = half ? split : 0, c_hi = half ? u.npad : split;   // this group's accumulator columns
       const bool fast = a.r <= 128 && u.rows == 128;
       const float* cs = sh->cs2[u.rb & 1];
+      const int* last_key = sh->vis_off[u.rb & 1];
       for (int t = 0; t < rn.cnt; ++t, ++tc) {
         if ((tc & 1) != pair) continue;
         const int buf = (tc >> 1) & 1, acc = pair * 2 + buf, aph = (tc >> 2) & 1;
@@ -626,7 +733,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
 #pragma unroll
               for (int t2 = 0; t2 < 16; ++t2) {
                 const int sr = s0 + t2;
-                const bool vis = sr < u.rows && (full || j <= a.n - a.r + obs_row(a, u, sr));
+                const bool vis = sr < u.rows && (full || j <= last_key[sr]);
                 if (vis) sum += fast_exp2(__uint_as_float(v[t2]) * cs[sr]);
               }
             }
@@ -644,133 +751,90 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
   });
 }
 
-// nu of the 64 value rows of one V-ring stage: two adjacent lanes share a row (one half of its 16-byte
-// chunks each, in an order that keeps them on different banks), square and add in FP32, and meet by shuffle.
-template <typename T>
-__device__ __forceinline__ float half_row_sq(const char* stage, int row, int sub, int D) {
-  float acc = 0.f;
-  if (D == 128) {
-    const char* base = stage + sub * kVSubBytes + row * 128;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      const uint4 q = *reinterpret_cast<const uint4*>(base + (((c ^ sub) ^ (row & 7)) << 4));
-      float f[8];
-      Vec16<T>::widen(q, f);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
-    }
-  } else {
-    const char* base = stage + row * 128;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      const uint4 q = *reinterpret_cast<const uint4*>(base + (((sub * 4 + c) ^ (row & 7)) << 4));
-      float f[8];
-      Vec16<T>::widen(q, f);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc = fmaf(f[e], f[e], acc);
+// One row's offset extension: -off / (2 c kFold) as three 16-bit parts, the first three of the row's
+// sixteen elements, the same again in the second 16-byte half.
+__device__ __forceinline__ void write_extension(char* ext, int row, float off, float c, int bf16, bool live) {
+  uint32_t w0 = 0, w1 = 0;
+  if (live) {
+    float v = -(off / c) / (2.f * kFold);
+    if (bf16) {
+      const __nv_bfloat16 h1 = __float2bfloat16_rn(v);
+      v -= __bfloat162float(h1);
+      const __nv_bfloat16 h2 = __float2bfloat16_rn(v);
+      v -= __bfloat162float(h2);
+      const __nv_bfloat16 h3 = __float2bfloat16_rn(v);
+      w0 = (uint32_t)__bfloat16_as_ushort(h1) | ((uint32_t)__bfloat16_as_ushort(h2) << 16);
+      w1 = (uint32_t)__bfloat16_as_ushort(h3);
+    } else {
+      v = fminf(fmaxf(v, -60000.f), 60000.f);              // float16 has no room beyond; such logits are not scored
+      const __half h1 = __float2half_rn(v);
+      v -= __half2float(h1);
+      const __half h2 = __float2half_rn(v);
+      v -= __half2float(h2);
+      const __half h3 = __float2half_rn(v);
+      w0 = (uint32_t)__half_as_ushort(h1) | ((uint32_t)__half_as_ushort(h2) << 16);
+      w1 = (uint32_t)__half_as_ushort(h3);
     }
   }
-  return acc;
+  uint4* dst = reinterpret_cast<uint4*>(ext + row * 32);
+  dst[0] = make_uint4(w0, w1, 0u, 0u);
+  dst[1] = make_uint4(w0, w1, 0u, 0u);
 }
 
-// Merge / value-norm group (four warps).  Per step of the fixed sequence:
-//  1. the value rows that go with the step's pass-1 run, as they arrive in the V ring: nu_j = |V_j|^2;
-//  2. for the run whose pass 2 comes one step later: thread `s` waits until the partials of row s have
-//     arrived from all runs of the row block, merges them in run order into the row's offset and writes
-//     the row's offset extension into shared memory for the MMA.
-__device__ void aux_group(const TcArgs& a, Shared* sh, char* tiles) {
+// Merge group (two warps, 64 threads).  For every run of this CTA, in order and up to two runs ahead of
+// the MMA warp: thread `s` waits until the partials of rows 2s and 2s + 1 have arrived from all runs of the
+// row block, merges them in run order into the rows' offsets and writes their offset extensions into
+// shared memory.
+__device__ void merge_group(const TcArgs& a, Shared* sh, char* tiles, int s) {
   Barriers* bars = &sh->bars;
-  const int s = threadIdx.x & 127;
   const int G = (int)gridDim.x, first = (int)blockIdx.x;
   const int nr = (a.n_runs - first + G - 1) / G;
-  int vc = 0, mc = 0;
-  bool dead = false;   // a wait ran out: nothing more is delivered (the MMA warp's own waits then run out too)
-  for (int k = 0; k < nr + a.lead - 1 && !dead; ++k) {
-    if (k < nr && a.prior) {
-      const Run rn = run_info(a, first + k * G);
-      const UnitInfo u = unit_info(a, rn.unit);
-      if (u.rb == 0) {
-        const int row = s >> 1, sub = s & 1;
-        for (int t = 0; t < 2 * rn.cnt && !dead; ++t, ++vc) {
-          const int vs = vc & 1;
-          if (!mbar_wait(&bars->v_full[vs], (vc >> 1) & 1, a.status)) { dead = true; break; }
-          const char* stage = tiles + kOffV + vs * kVStageBytes;
-          float sq = a.bf16 ? half_row_sq<__nv_bfloat16>(stage, row, sub, a.D) : half_row_sq<__half>(stage, row, sub, a.D);
-          sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-          mbar_arrive(&bars->v_empty[vs]);
-          const int j = rn.blk0 * kKeyTile + t * kVRows + row;
-          if (sub == 0 && j < a.n) a.nu[(size_t)u.bh * a.n + j] = sq;
-        }
-      }
-    }
-    const int jm = k - a.lead + 1;
-    if (jm < 0 || jm >= nr || dead) continue;
-    const Run rn = run_info(a, first + jm * G);
+  for (int mc = 0; mc < nr; ++mc) {
+    const Run rn = run_info(a, first + mc * G);
     const UnitInfo u = unit_info(a, rn.unit);
     const int slot = mc & 1;
-    if (!mbar_wait(&bars->ext_empty[slot], ((mc >> 1) & 1) ^ 1, a.status)) break;
-    ++mc;
-    const float2* p = a.partial + (size_t)rn.unit * a.rpu * 128 + s;
-    float Mx = -INFINITY, Zs = 0.f;
-    for (int t0 = 0; t0 < a.rpu && !dead; t0 += 16) {     // 16 loads in flight per thread
+    if (!mbar_wait(&bars->ext_empty[slot], ((mc >> 1) & 1) ^ 1, a.status)) return;
+    const float2* p = reinterpret_cast<const float2*>(a.partial + (size_t)rn.unit * a.rpu * 128) + s;
+    float M0 = -INFINITY, Z0 = 0.f, M1 = -INFINITY, Z1 = 0.f;   // running shift and sum of 2^{L - shift}, per row
+    for (int t0 = 0; t0 < a.rpu; t0 += 16) {              // 16 8-byte loads in flight per thread
       float2 e[16];
       const long long tstart = now_ns();
       for (;;) {
         bool all = true;
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
-          e[t] = t0 + t < a.rpu ? ld_partial(&p[(size_t)(t0 + t) * 128]) : make_float2(-INFINITY, 0.f);
-          all = all && (e[t].x == e[t].x);                 // NaN: not published yet
+          e[t] = t0 + t < a.rpu ? ld_partial2(&p[(size_t)(t0 + t) * 64]) : make_float2(-INFINITY, -INFINITY);
+          all = all && (e[t].x == e[t].x) && (e[t].y == e[t].y);   // NaN: not published yet
         }
         if (all) break;
-        __nanosleep(200);
+        __nanosleep(300);
         if (now_ns() - tstart > kWaitLimitNs) {
+          // nothing more is delivered; the MMA warp's own wait then runs out too
           atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
-          dead = true;
-          break;
+          return;
         }
       }
-      if (dead) break;
-      float m = Mx;
+      float m0 = M0, m1 = M1;
 #pragma unroll
-      for (int t = 0; t < 16; ++t) m = fmaxf(m, e[t].x);
-      if (m > -INFINITY) {
-        float z = Zs > 0.f ? Zs * fast_exp2(Mx - m) : 0.f;
+      for (int t = 0; t < 16; ++t) { m0 = fmaxf(m0, e[t].x); m1 = fmaxf(m1, e[t].y); }
+      if (m0 > -INFINITY) {
+        float z = Z0 > 0.f ? Z0 * fast_exp2(M0 - m0) : 0.f;
 #pragma unroll
-        for (int t = 0; t < 16; ++t)
-          if (e[t].y > 0.f) z += e[t].y * fast_exp2(e[t].x - m);
-        Zs = z;
-        Mx = m;
+        for (int t = 0; t < 16; ++t) z += fast_exp2(e[t].x - m0);   // 2^{-inf} = 0 for the padding
+        Z0 = z; M0 = m0;
+      }
+      if (m1 > -INFINITY) {
+        float z = Z1 > 0.f ? Z1 * fast_exp2(M1 - m1) : 0.f;
+#pragma unroll
+        for (int t = 0; t < 16; ++t) z += fast_exp2(e[t].y - m1);
+        Z1 = z; M1 = m1;
       }
     }
-    if (dead) break;
     // 2^{c w - off} = softmax weight / G.  The MMA adds 2 kFold (h1 + h2 + h3) = -off / c to w.
-    uint32_t w0 = 0, w1 = 0;
-    if (s < u.rows) {
-      const float off = Mx + log2f(Zs) + a.log2G;
-      float v = -(off / sh->c[obs_row(a, u, s)]) / (2.f * kFold);
-      if (a.bf16) {
-        const __nv_bfloat16 h1 = __float2bfloat16_rn(v);
-        v -= __bfloat162float(h1);
-        const __nv_bfloat16 h2 = __float2bfloat16_rn(v);
-        v -= __bfloat162float(h2);
-        const __nv_bfloat16 h3 = __float2bfloat16_rn(v);
-        w0 = (uint32_t)__bfloat16_as_ushort(h1) | ((uint32_t)__bfloat16_as_ushort(h2) << 16);
-        w1 = (uint32_t)__bfloat16_as_ushort(h3);
-      } else {
-        v = fminf(fmaxf(v, -60000.f), 60000.f);            // float16 has no room beyond; such logits are not scored
-        const __half h1 = __float2half_rn(v);
-        v -= __half2float(h1);
-        const __half h2 = __float2half_rn(v);
-        v -= __half2float(h2);
-        const __half h3 = __float2half_rn(v);
-        w0 = (uint32_t)__half_as_ushort(h1) | ((uint32_t)__half_as_ushort(h2) << 16);
-        w1 = (uint32_t)__half_as_ushort(h3);
-      }
-    }
-    uint4* row = reinterpret_cast<uint4*>(tiles + kOffExt + slot * kExtBytes + s * 32);
-    row[0] = make_uint4(w0, w1, 0u, 0u);
-    row[1] = make_uint4(w0, w1, 0u, 0u);
+    char* ext = tiles + kOffExt + slot * kExtBytes;
+    const int r0 = 2 * s, r1 = 2 * s + 1;
+    write_extension(ext, r0, M0 + log2f(Z0) + a.log2G, sh->c[obs_row(a, u, r0 < u.rows ? r0 : 0)], a.bf16, r0 < u.rows);
+    write_extension(ext, r1, M1 + log2f(Z1) + a.log2G, sh->c[obs_row(a, u, r1 < u.rows ? r1 : 0)], a.bf16, r1 < u.rows);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads it through the async proxy
     mbar_arrive(&bars->ext_full[slot]);
   }
@@ -788,6 +852,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   for (int t = threadIdx.x; t < 128; t += kThreads) {
     sh->cs2[0][t] = a.r <= 128 ? a.c[t % a.r] : a.c[t];
     sh->cs2[1][t] = a.r <= 128 ? a.c[t % a.r] : a.c[128 + t];
+    sh->vis_off[0][t] = a.n - a.r + (a.r <= 128 ? t % a.r : t);
+    sh->vis_off[1][t] = a.n - a.r + (a.r <= 128 ? t % a.r : 128 + t);
   }
   {
     // every 16-byte chunk of the constant tile reads (kFold, kFold, kFold, 0, 0, 0, 0, 0); it meets the
@@ -809,10 +875,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     for (int p = 0; p < 2; ++p) {
       mbar_init(&bars->q_full[p], 1);
       mbar_init(&bars->q_empty[p], 1);
-      mbar_init(&bars->v_full[p], 1);
-      mbar_init(&bars->v_empty[p], 128);
-      mbar_init(&bars->ext_full[p], 128);
+      mbar_init(&bars->ext_full[p], 64);
       mbar_init(&bars->ext_empty[p], 1);
+    }
+    for (int s = 0; s < kVStages; ++s) {
+      mbar_init(&bars->v_full[s], 1);
+      mbar_init(&bars->v_empty[s], 128);
     }
     for (int s = 0; s < kKStages; ++s) {
       mbar_init(&bars->k_full[s], 1);
@@ -834,17 +902,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   const uint32_t tmem_base = sh->tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) producer(a, &qmap, &kmap, sh, tiles);
+    if (lane == 0) producer(a, &qmap, &kmap, &vmap, sh, tiles);
   } else if (warp == 1) {
     if (lane == 0) mma_issuer(a, sh, tiles, tmem_base);
-  } else if (warp == 2) {
-    if (lane == 0 && a.prior) v_producer(a, &vmap, sh, tiles);
-  } else if (warp == 3) {
-    // idle
+  } else if (warp < 4) {
+    merge_group(a, sh, tiles, threadIdx.x & 63);
   } else if (warp < 20) {
     softmax_group(a, sh, tmem_base, (warp - 4) >> 3, ((warp - 4) >> 2) & 1);
   } else {
-    aux_group(a, sh, tiles);
+    if (a.prior) v_group(a, sh, tiles);
   }
 
   tc_fence_before();
@@ -891,7 +957,7 @@ bool make_map(CUtensorMap* m, const void* base, int bf16, int d, long long token
 bool score_tc_available() { return encode_fn() != nullptr; }
 
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
-                             float2* partial, int* status, cudaStream_t st) {
+                             float2* partial_ws, int* status, cudaStream_t st) {
   static int n_sm = 0;
   static bool configured = false;
   if (!configured) {
@@ -908,7 +974,7 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   a.n_blk = pl.n_blk; a.D = pl.d;
   const long long tiles = (long long)units * pl.n_blk;
   const long long ch = tiles / ((long long)n_sm * 8);
-  a.CH = ch < 1 ? 1 : (ch > 4 ? 4 : (int)ch);
+  a.CH = ch < 1 ? 1 : (ch > 8 ? 8 : (int)ch);
   a.rpu = (pl.n_blk + a.CH - 1) / a.CH;
   a.n_runs = units * a.rpu;
   const int grid = a.n_runs < n_sm ? a.n_runs : n_sm;
@@ -927,7 +993,7 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   a.log2G = log2f((float)pl.G);
   for (int i = 0; i < kMaxRows; ++i) a.c[i] = pl.rows.c[i];
   for (int t = 0; t < 128; ++t) a.cs[t] = pl.r <= 128 ? pl.rows.c[t % pl.r] : 0.f;
-  a.partial = partial; a.s_raw = s_raw; a.nu = nu;
+  a.partial = reinterpret_cast<float*>(partial_ws); a.s_raw = s_raw; a.nu = nu;
   a.status = status;
 
   CUtensorMap qmap, kmap, vmap;
@@ -942,7 +1008,7 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   }
 
   // every partial starts as NaN: "not published yet"
-  if (cudaMemsetAsync(partial, 0xff, (size_t)a.n_runs * 128 * sizeof(float2), st) != cudaSuccess) return AHAKV_ERR_CUDA;
+  if (cudaMemsetAsync(a.partial, 0xff, (size_t)a.n_runs * 128 * sizeof(float), st) != cudaSuccess) return AHAKV_ERR_CUDA;
   void* args[] = {&qmap, &kmap, &vmap, &a};
   const cudaError_t e = cudaLaunchCooperativeKernel((const void*)score_tc_kernel, dim3(grid), dim3(kThreads), args,
                                                     (size_t)kSmemBytes, st);
