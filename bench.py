@@ -59,8 +59,11 @@ def algorithmic_work(w):
     q_read = w.batch * w.n_q_heads * w.obs_window * w.head_dim * es
     kv_write = 2 * w.batch * w.n_kv_heads * w.n_keep * w.head_dim * es
     flops = 2 * w.batch * w.n_q_heads * w.obs_window * w.n_ctx * w.head_dim
-    return dict(bytes=kv_read + q_read + kv_write, flops=flops,
-                score_bytes=kv_read // 2 + q_read + 4 * w.batch * w.n_kv_heads * w.n_ctx)
+    # the scoring kernel: K once and, with the value prior, V once (its value-norm warps), Q_obs, and the
+    # raw score and nu vectors it writes (4 bytes per token and KV head each)
+    per_token = 4 * w.batch * w.n_kv_heads * w.n_ctx
+    score_bytes = kv_read // 2 + q_read + per_token + ((kv_read // 2 + per_token) if w.value_prior else 0)
+    return dict(bytes=kv_read + q_read + kv_write, flops=flops, score_bytes=score_bytes)
 
 
 class ClockSampler:
@@ -309,13 +312,17 @@ def run_ours(args):
     t_roof_ms = 1e3 * max(work["flops"] / (pk["bf16_tflops_sustained"] * 1e12), work["bytes"] / (pk["hbm_gbs"] * 1e9))
     top = max(stage_ms, key=stage_ms.get)
     stage_bytes = {"score": work["score_bytes"],
-                   "vnorm": w.batch * w.n_kv_heads * w.n_ctx * (w.head_dim * w.elem_size + 4),
                    "compact": 2 * 2 * w.batch * w.n_kv_heads * w.n_keep * w.head_dim * w.elem_size}
     dom = "score"
     achieved = stage_bytes[dom] / (stage_ms[dom] * 1e-3) / 1e9 if stage_ms[dom] > 0 else 0.0
-    roofline = {"kernel": "scoring kernels (logits, SG-softmax, column sums)", "bound": "hbm",
+    # DRAM bytes of one launch from the ncu capture summarised in profiles/score_tc_kernel_long32k_b2.txt:
+    # 1117.8 MB at batch 2, scaled by the units a launch of this run processes (traffic grows with them).
+    traffic = None
+    if w.name == "long_32k" and w.value_prior:
+        traffic = 1117.8e6 * w.batch / 2
+    roofline = {"kernel": "score_tc_kernel (logits, SG-softmax, column sums, value norms)", "bound": "hbm",
                 "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
-                "peak_source": f"{pk['source']} (sustained copy)", "traffic": None,
+                "peak_source": f"{pk['source']} (sustained copy)", "traffic": traffic,
                 "algorithmic_bytes_per_launch": stage_bytes[dom], "ms_per_launch": stage_ms[dom],
                 "slowest_stage": top}
     out = {
