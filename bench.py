@@ -110,6 +110,23 @@ class ClockSampler:
                     samples=len(sm), reasons=sorted(reasons))
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: what a multi-GPU number is divided by (no other data-path collective exists)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_step: int, world: int, ms_step: float) -> float:
+    """Replicas only: every rank evicts its own layer, so the job's throughput is world x one replica's
+    tokens over the slowest rank's time."""
+    return world * tokens_per_step / (ms_step * 1e-3)
+
+
 def cpu_oracle_sample(w, seconds_hint=15.0):
     """Times the oracle, as it stands, on a bounded sample of the workload: whole (sequence, KV head)
     units of layer 0, one per host thread per round.  Returns (tokens/s for a full layer, info)."""
@@ -252,13 +269,10 @@ def run_ours(args):
     launches = ab.ahakv_launch_count() - launches0
     clocks = sampler.stop() if sampler else None
     status = ab.ahakv_last_device_status(ws)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
     tokens_per_step = w.batch * w.n_ctx
-    value = world * tokens_per_step / (ms_step * 1e-3)
+    value = whole_job_value(tokens_per_step, world, ms_step)
 
     # ---- per-stage device times over the same K steps (events inside the library) ----------------------
     ab.ahakv_profile_enable(True)
@@ -291,13 +305,10 @@ def run_ours(args):
         a1.record(stream)
         barrier()
         e2e_ms = a0.elapsed_time(a1) / args.e2e_steps
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e2e_ms, world, dev)
         h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
         d2h = sum(t.numel() * t.element_size() for t in houts)
-        e2e = {"value": world * tokens_per_step / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": whole_job_value(tokens_per_step, world, e2e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": args.e2e_steps,
                "api": "ahakv_evict through the C ABI, pinned host buffers copied in and out every step"}
         del hq, hk, hv, dq, dk, dv, houts
