@@ -44,7 +44,7 @@ ahakv_status launch_score_simt(const Plan& pl, const void* q, const void* k, flo
                                float* final_off, cudaStream_t st);
 // Also streams V and writes nu when the value prior is on (v and nu non-null).
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
-                             float2* partial, int* status, cudaStream_t st);
+                             float2* partial, int* counters, int* status, cudaStream_t st);
 bool score_tc_available();
 ahakv_status launch_vnorm(const Plan& pl, const void* v, float* nu, cudaStream_t st);
 ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,

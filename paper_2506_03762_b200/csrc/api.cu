@@ -133,7 +133,8 @@ static ahakv_status queue_score(const Plan& pl, const void* q, const void* k, co
   const bool prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0;
   float* nu = prior ? at<float>(ws, pl.off_nu) : nullptr;
   if (pl.use_tc)   // the tensor-core kernel squares the value rows on its way
-    rc = launch_score_tc(pl, q, k, prior ? v : nullptr, s_raw, nu, partial, at<int>(ws, pl.off_status), st);
+    rc = launch_score_tc(pl, q, k, prior ? v : nullptr, s_raw, nu, partial, at<int>(ws, pl.off_sync),
+                         at<int>(ws, pl.off_status), st);
   else
     rc = launch_score_simt(pl, q, k, s_raw, partial, final_off, st);
   if (rc) return rc;

@@ -18,14 +18,16 @@
 // TMA (128-byte swizzle) from the same K-major Q and K tiles, which serve as A or
 // B operand alike.
 //
-// Schedule.  A run is up to CH consecutive key tiles of one row block; run q belongs
-// to CTA q mod grid.  Every CTA walks ONE fixed sequence of segments,
-//     P1(run 0) .. P1(run lead-1), then P1(run i+lead), P2(run i), P1(run i+lead+1), P2(run i+1), ..
-// through one pipeline: one TMA warp, one MMA warp, a ring of K tiles, four TMEM
-// accumulators and sixteen softmax warps that take whichever kind of tile comes
-// next.  Pass 2 of a run thus trails its pass 1 by `lead` steps: long enough for
-// every CTA to have delivered its share of the row block's statistics, short
-// enough for the keys to be still in L2, so that HBM sees K once.
+// Schedule.  A run is up to CH consecutive key tiles of one row block.  Runs are handed out to the CTAs
+// as they come free, from two global counters: one for pass 1, one for pass 2.  The TMA thread of
+// every CTA takes one run of each per round (pass 2 only once every pass-1 run of that row block has been
+// taken by somebody) and publishes the CTA's sequence of segments, P1(a), P2(b), P1(a'), P2(b'), ..., in a
+// ring in shared memory that all other roles read in order; the pass-2 run of a round is announced to the
+// merge group a round early.  One pipeline serves the sequence: one TMA warp, one MMA warp, a ring of K
+// tiles, four TMEM accumulators and sixteen softmax warps that take whichever kind of tile comes next.
+// Pass 2 trails pass 1 by about one round of the whole grid: long enough for every CTA to have delivered
+// its share of a row block's statistics, short enough for the keys to be still in L2, so that HBM sees K
+// once.  SMs that fall behind simply take fewer runs.
 //
 // Between the passes there are no flags, counters or fences.  The partials start
 // as NaN (the host clears them before the launch) and each is published by a single
@@ -49,8 +51,8 @@
 // launch and no second sweep of HBM.
 //
 // The kernel is launched cooperatively with at most one CTA per SM, which guarantees
-// that the CTAs a partial comes from are running; a wait only ever depends on work
-// that is earlier in the fixed sequence, so the waits cannot deadlock.  Every wait is
+// that the CTAs a partial comes from are running; a segment only ever waits for
+// segments that were handed out before it, so the waits cannot deadlock.  Every wait is
 // bounded in time; on expiry the kernel records AHAKV_ERR_TIMEOUT in the status word
 // and winds down.
 #include <cuda.h>
@@ -64,8 +66,12 @@ constexpr int kKStages = 3;                // K-tile ring depth
 constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 16-bit elements, 128-byte swizzled
 constexpr int kVRows = 64;                 // value rows per V-ring stage
 constexpr int kVStages = 2;
+constexpr int kSegRing = 64;               // published segments a role may lag behind the scheduler
+constexpr int kMergeRing = 8;
+constexpr int kSegAhead = 4;               // segments published beyond the one the softmax warps are on
+constexpr int kSegEnd = -1;
 constexpr int kVSubBytes = kVRows * 128;
-constexpr int kThreads = 768;              // TMA warp, MMA warp, 2 merge warps, 16 softmax warps, 4 value-norm warps
+constexpr int kThreads = 768;              // TMA + scheduler warp, MMA warp, 2 merge warps, 16 softmax warps, 4 value-norm warps
 constexpr long long kWaitLimitNs = 1000000000LL;   // 1 s
 constexpr float kFold = 256.f;             // value of the constant tile; offsets are stored divided by it
 
@@ -74,7 +80,6 @@ struct TcArgs {
   int CH;         // key tiles per run
   int rpu;        // runs per row block = ceil(n_blk / CH)
   int n_runs;     // row blocks * rpu
-  int lead;       // pass 2 of a run comes `lead` steps after its pass 1
   int bf16;       // operand type of the products
   int prior;      // stream V and write nu
   float log2G;
@@ -83,6 +88,7 @@ struct TcArgs {
   float* partial;    // [unit][run][128]: log2 of a row's sum of 2^{c w} over the run's keys
   float* s_raw;      // [unit][n]
   float* nu;         // [B * Hkv][n]
+  int* ctr;          // [2] next pass-1 run, next pass-2 run (zero at launch)
   int* status;
 };
 
@@ -98,7 +104,10 @@ struct __align__(8) Barriers {
 struct Shared {
   Barriers bars;
   uint32_t tmem_slot;
-  int pad_;
+  int seg_pub, seg_done_soft, seg_done_v;   // segments published / retired by the softmax warps / by the value-norm warps
+  int mrg_pub, mrg_done;                    // pass-2 runs announced to / finished by the merge group
+  int seg[kSegRing];                        // 2 * run + pass, or kSegEnd
+  int mrg[kMergeRing];                      // run, or kSegEnd
   float c[kMaxRows];            // lambda_i * log2(e) per observation row
   float cs2[2][128];            // c per stacked row, by row block parity (r > 128 has two kinds of block)
   int vis_off[2][128];          // per stacked row: n - r + its observation row = the last key it may see
@@ -316,61 +325,131 @@ __device__ __forceinline__ unsigned long long policy_evict_first() {
   return p;
 }
 
-// The fixed sequence of segments of this CTA: f(pass, run) for P1(0) .. P1(lead-1), then alternately
-// P1(i + lead), P2(i).  Every role walks it with the same counters.
-template <typename F>
-__device__ __forceinline__ void for_each_segment(const TcArgs& a, F f) {
-  const int G = (int)gridDim.x, first = (int)blockIdx.x;
-  const int nr = (a.n_runs - first + G - 1) / G;
-  for (int k = 0; k < nr + a.lead; ++k) {
-    if (k < nr) f(0, first + k * G);
-    if (k >= a.lead) f(1, first + (k - a.lead) * G);
-  }
-}
+// ---- the CTA's sequence of segments -------------------------------------------------------------------
+__device__ __forceinline__ int ld_volatile(const int* p) { return *(const volatile int*)p; }
 
-// The fixed sequence again, as a cursor that can be advanced one segment at a time.
-struct SegCursor {
-  int k, sub;
-};
-__device__ __forceinline__ bool seg_next(const TcArgs& a, int nr, SegCursor& c, int& pass, int& run) {
-  const int G = (int)gridDim.x, first = (int)blockIdx.x;
-  while (c.k < nr + a.lead) {
-    if (c.sub == 0) {
-      c.sub = 1;
-      if (c.k < nr) { pass = 0; run = first + c.k * G; return true; }
+// Entry `idx` of the sequence if the scheduler has published it, else -2.
+__device__ __forceinline__ int seg_peek(Shared* sh, int idx) {
+  if (idx >= ld_volatile(&sh->seg_pub)) return -2;
+  __threadfence_block();
+  return ld_volatile(&sh->seg[idx % kSegRing]);
+}
+// The same, waiting (bounded) for the scheduler.  kSegEnd ends the sequence; so does a wait that ran out.
+__device__ __forceinline__ int seg_get(Shared* sh, int idx, int* status) {
+  int e = seg_peek(sh, idx);
+  if (e != -2) return e;
+  const long long t0 = now_ns();
+  for (;;) {
+    __nanosleep(64);
+    if ((e = seg_peek(sh, idx)) != -2) return e;
+    if (now_ns() - t0 > kWaitLimitNs) {
+      atomicExch(status, (int)AHAKV_ERR_TIMEOUT);
+      return kSegEnd;
     }
-    c.sub = 0;
-    const int k = c.k++;
-    if (k >= a.lead) { pass = 1; run = first + (k - a.lead) * G; return true; }
   }
-  return false;
+}
+__device__ __forceinline__ int mrg_get(Shared* sh, int idx, int* status) {
+  const long long t0 = now_ns();
+  for (;;) {
+    if (idx < ld_volatile(&sh->mrg_pub)) {
+      __threadfence_block();
+      return ld_volatile(&sh->mrg[idx % kMergeRing]);
+    }
+    __nanosleep(200);
+    if (now_ns() - t0 > kWaitLimitNs) {
+      atomicExch(status, (int)AHAKV_ERR_TIMEOUT);
+      return kSegEnd;
+    }
+  }
 }
 
-// The next 64 value rows to fetch or to square: stage t of the run at step k (first row block of a KV
-// head only).
-struct VCursor {
-  int k, t, cnt, row0, b, h, bh;
+// f(pass, run) for every segment of this CTA, in order.
+template <typename F>
+__device__ __forceinline__ void for_each_segment(const TcArgs& a, Shared* sh, F f) {
+  for (int idx = 0;; ++idx) {
+    const int e = seg_get(sh, idx, a.status);
+    if (e == kSegEnd) return;
+    f(e & 1, e >> 1, idx);
+  }
+}
+
+// Scheduler state of a CTA (kept by its TMA thread): hands the CTA its runs.  A round takes the next pass-1
+// run and publishes it; publishes the pass-2 run taken in an earlier round -- only once every pass-1 run of
+// its row block has been taken by somebody, so that whoever waits for that block's statistics waits for work
+// that is already under way; then takes the next pass-2 run and announces it to the merge group.
+struct Scheduler {
+  int k, m, pend;
+  bool p1_left, p2_left, done;
 };
-__device__ __forceinline__ bool v_seek(const TcArgs& a, int nr, VCursor& c) {
-  const int G = (int)gridDim.x, first = (int)blockIdx.x;
-  for (; c.k < nr; ++c.k) {
-    const Run rn = run_info(a, first + c.k * G);
+__device__ __forceinline__ void sched_publish(Shared* sh, Scheduler& sc, int entry) {
+  sh->seg[sc.k % kSegRing] = entry;
+  __threadfence_block();
+  *(volatile int*)&sh->seg_pub = ++sc.k;
+}
+__device__ __forceinline__ void sched_announce(Shared* sh, Scheduler& sc, int run) {
+  sh->mrg[sc.m % kMergeRing] = run;
+  __threadfence_block();
+  *(volatile int*)&sh->mrg_pub = ++sc.m;
+}
+// One round, if there is room for it (never waits).  Returns whether anything was published.
+__device__ bool sched_round(const TcArgs& a, Shared* sh, Scheduler& sc) {
+  if (sc.done) return false;
+  const int ds = ld_volatile(&sh->seg_done_soft), dv = ld_volatile(&sh->seg_done_v);
+  // room in both rings for a whole round, and not too far ahead of the tiles being worked on
+  if (sc.k - (ds < dv ? ds : dv) > kSegRing - 4 || sc.k - ds >= kSegAhead ||
+      sc.m - ld_volatile(&sh->mrg_done) > kMergeRing - 2)
+    return false;
+  bool did = false;
+  if (sc.p1_left) {
+    const int r = atomicAdd(&a.ctr[0], 1);
+    if (r < a.n_runs) { sched_publish(sh, sc, 2 * r); did = true; }
+    else sc.p1_left = false;
+  }
+  if (sc.pend >= 0) {
+    // the pass-2 run in hand joins the sequence once all pass-1 runs of its row block have been taken
+    const int need = min((sc.pend / a.rpu + 1) * a.rpu, a.n_runs);
+    if (ld_volatile(&a.ctr[0]) >= need) { sched_publish(sh, sc, 2 * sc.pend + 1); sc.pend = -1; did = true; }
+  }
+  if (sc.pend < 0 && sc.p2_left) {
+    const int b = atomicAdd(&a.ctr[1], 1);
+    if (b < a.n_runs) { sc.pend = b; sched_announce(sh, sc, b); did = true; }
+    else sc.p2_left = false;
+  }
+  if (!sc.p1_left && !sc.p2_left && sc.pend < 0) {
+    sched_announce(sh, sc, kSegEnd);
+    sched_publish(sh, sc, kSegEnd);
+    sc.done = true;
+    did = true;
+  }
+  return did;
+}
+
+// The next 64 value rows to fetch or to square: stage t of a pass-1 segment (first row block of a KV head
+// only).  `idx` walks the CTA's sequence.
+struct VCursor {
+  int idx, t, cnt, row0, b, h, bh;
+};
+// Moves to the first stage of the next segment that brings value rows.  1: found, 0: the sequence has ended,
+// -1: not published yet (only when `block` is false).
+__device__ __forceinline__ int v_seek(const TcArgs& a, Shared* sh, VCursor& c, bool block, int* behind = nullptr) {
+  for (;; ++c.idx) {
+    if (behind) *(volatile int*)behind = c.idx;               // everything before c.idx has been dealt with
+    const int e = block ? seg_get(sh, c.idx, a.status) : seg_peek(sh, c.idx);
+    if (e == -2) return -1;
+    if (e == kSegEnd) return 0;
+    if (e & 1) continue;
+    const Run rn = run_info(a, e >> 1);
     const UnitInfo u = unit_info(a, rn.unit);
     if (u.rb != 0) continue;
     c.t = 0; c.cnt = 2 * rn.cnt; c.row0 = rn.blk0 * kKeyTile; c.b = u.b; c.h = u.h; c.bh = u.bh;
-    return true;
+    return 1;
   }
-  return false;
-}
-__device__ __forceinline__ bool v_advance(const TcArgs& a, int nr, VCursor& c) {
-  if (++c.t < c.cnt) return true;
-  ++c.k;
-  return v_seek(a, nr, c);
 }
 
 // ---- roles --------------------------------------------------------------------------------------------
-// TMA producer: one thread feeds two independent streams, whichever has a free slot: Q and K tiles in
-// the order of the fixed sequence, and the value rows that go with the pass-1 key tiles.
+// TMA producer: one thread keeps the CTA's sequence of segments filled (scheduler rounds) and feeds two
+// independent streams, whichever has a free slot: Q and K tiles in the order of the sequence, and the value
+// rows that go with the pass-1 key tiles.
 __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, const CUtensorMap* vmap,
                          Shared* sh, char* tiles) {
   Barriers* bars = &sh->bars;
@@ -378,61 +457,69 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
   const int q_rows = a.r <= 128 ? a.hb * a.r : 128;
   const int q_bytes = n_sub * q_rows * 128, k_bytes = n_sub * kSubTileBytes;
   const unsigned long long once = policy_evict_first();
-  const int G = (int)gridDim.x, first = (int)blockIdx.x;
-  const int nr = (a.n_runs - first + G - 1) / G;
 
-  // K stream state
-  SegCursor sc_cur = {0, 0};
-  int pass = 0, run = 0, tc = 0, sc = 0, t = 0;
-  Run rn = run_info(a, first);
-  UnitInfo u = unit_info(a, rn.unit);
-  bool k_live = seg_next(a, nr, sc_cur, pass, run), q_due = true;
-  if (k_live) { rn = run_info(a, run); u = unit_info(a, rn.unit); }
-  // V stream state
+  // K stream state: 0 waiting for the next segment, 1 Q to load, 2 tiles to load, 3 done
+  int k_state = 0, k_idx = 0, pass = 0, tc = 0, sc = 0, t = 0;
+  Run rn = run_info(a, 0);
+  UnitInfo u = unit_info(a, 0);
+  // V stream state: 0 waiting for the next segment with value rows, 2 stages to load, 3 done
   VCursor vcur;
-  vcur.k = 0;
-  bool v_live = a.prior && v_seek(a, nr, vcur);
-  int vc = 0;
+  vcur.idx = 0;
+  int v_state = a.prior ? 0 : 3, vc = 0;
 
+  Scheduler sched = {0, 0, -1, true, true, false};
   long long idle_since = -1;
-  while (k_live || v_live) {
+  while (k_state != 3 || v_state != 3) {
     bool progress = false;
-    if (k_live) {
-      if (q_due) {
-        const int qb = sc & 1;
-        if (mbar_try(&bars->q_empty[qb], ((sc >> 1) & 1) ^ 1)) {
-          char* q_smem = tiles + kOffQ + qb * kQBytes;
-          mbar_expect_tx(&bars->q_full[qb], q_bytes);
-          for (int s = 0; s < n_sub; ++s) {
-            if (a.r <= 128) tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, 0, u.h * a.G + u.rb * a.hb, u.b);
-            else tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, u.rb * 128, u.h, u.b);
-          }
-          ++sc;
-          q_due = false;
-          progress = true;
-        }
-      } else {
-        const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
-        if (mbar_try(&bars->k_empty[stage], ph ^ 1)) {
-          mbar_expect_tx(&bars->k_full[stage], k_bytes);
-          char* dst = tiles + kOffK + stage * kKStageBytes;
-          for (int s = 0; s < n_sub; ++s) {
-            // the second read of a key tile is its last: let L2 drop it first
-            if (pass == 0) tma_load_4d(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b);
-            else tma_load_4d_hint(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b, once);
-          }
-          ++tc;
-          if (++t == rn.cnt) {
-            t = 0;
-            q_due = true;
-            k_live = seg_next(a, nr, sc_cur, pass, run);
-            if (k_live) { rn = run_info(a, run); u = unit_info(a, rn.unit); }
-          }
-          progress = true;
-        }
+    // a new round whenever the K stream is about to run dry
+    if (k_state == 0 && seg_peek(sh, k_idx) == -2) progress = sched_round(a, sh, sched);
+    if (k_state == 0) {
+      const int e = seg_peek(sh, k_idx);
+      if (e == kSegEnd) { k_state = 3; progress = true; }
+      else if (e != -2) {
+        ++k_idx;
+        pass = e & 1;
+        rn = run_info(a, e >> 1);
+        u = unit_info(a, rn.unit);
+        t = 0;
+        k_state = 1;
+        progress = true;
       }
     }
-    if (v_live) {
+    if (k_state == 1) {
+      const int qb = sc & 1;
+      if (mbar_try(&bars->q_empty[qb], ((sc >> 1) & 1) ^ 1)) {
+        char* q_smem = tiles + kOffQ + qb * kQBytes;
+        mbar_expect_tx(&bars->q_full[qb], q_bytes);
+        for (int s = 0; s < n_sub; ++s) {
+          if (a.r <= 128) tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, 0, u.h * a.G + u.rb * a.hb, u.b);
+          else tma_load_4d(q_smem + s * kSubTileBytes, qmap, &bars->q_full[qb], s * 64, u.rb * 128, u.h, u.b);
+        }
+        ++sc;
+        k_state = 2;
+        progress = true;
+      }
+    } else if (k_state == 2) {
+      const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
+      if (mbar_try(&bars->k_empty[stage], ph ^ 1)) {
+        mbar_expect_tx(&bars->k_full[stage], k_bytes);
+        char* dst = tiles + kOffK + stage * kKStageBytes;
+        for (int s = 0; s < n_sub; ++s) {
+          // the second read of a key tile is its last: let L2 drop it first
+          if (pass == 0) tma_load_4d(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b);
+          else tma_load_4d_hint(dst + s * kSubTileBytes, kmap, &bars->k_full[stage], s * 64, (rn.blk0 + t) * kKeyTile, u.h, u.b, once);
+        }
+        ++tc;
+        if (++t == rn.cnt) k_state = 0;
+        progress = true;
+      }
+    }
+    if (v_state == 0) {
+      const int f = v_seek(a, sh, vcur, false);
+      if (f == 1) { v_state = 2; progress = true; }
+      else if (f == 0) { v_state = 3; progress = true; }
+    }
+    if (v_state == 2) {
       const int vs = vc % kVStages;
       if (mbar_try(&bars->v_empty[vs], ((vc / kVStages) & 1) ^ 1)) {
         mbar_expect_tx(&bars->v_full[vs], n_sub * kVSubBytes);
@@ -440,7 +527,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
         for (int s = 0; s < n_sub; ++s)
           tma_load_4d_hint(dst + s * kVSubBytes, vmap, &bars->v_full[vs], s * 64, vcur.row0 + vcur.t * kVRows, vcur.h, vcur.b, once);
         ++vc;
-        v_live = v_advance(a, nr, vcur);
+        if (++vcur.t == vcur.cnt) { ++vcur.idx; v_state = 0; }
         progress = true;
       }
     }
@@ -451,6 +538,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
       if (idle_since < 0) idle_since = now;
       else if (now - idle_since > kWaitLimitNs) {
         atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
+        if (!sched.done) { sched_announce(sh, sched, kSegEnd); sched_publish(sh, sched, kSegEnd); }
         // wind down: give copies already in flight a bounded time (1 ms) to land before the CTA exits
         while (now_ns() - now < 1000000) __nanosleep(1000);
         return;
@@ -465,38 +553,40 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
 __device__ void v_group(const TcArgs& a, Shared* sh, char* tiles) {
   Barriers* bars = &sh->bars;
   const int row = (threadIdx.x & 127) >> 1, sub = threadIdx.x & 1;
-  const int G = (int)gridDim.x, first = (int)blockIdx.x;
-  const int nr = (a.n_runs - first + G - 1) / G;
+  const bool leader = (threadIdx.x & 127) == 0;
   VCursor cc;
-  cc.k = 0;
-  bool cv = v_seek(a, nr, cc);
-  for (int ci = 0; cv; ++ci) {
-    const int vs = ci % kVStages;
-    if (!mbar_wait(&bars->v_full[vs], (ci / kVStages) & 1, a.status)) return;
-    const char* stage = tiles + kOffV + vs * kVStageBytes;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+  cc.idx = 0;
+  int ci = 0;
+  while (v_seek(a, sh, cc, true, leader ? &sh->seg_done_v : nullptr) == 1) {
+    for (; cc.t < cc.cnt; ++cc.t, ++ci) {
+      const int vs = ci % kVStages;
+      if (!mbar_wait(&bars->v_full[vs], (ci / kVStages) & 1, a.status)) return;
+      const char* stage = tiles + kOffV + vs * kVStageBytes;
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int c = 0; c < 8; ++c) {
-      // head_dim 128: lane `sub` takes sub-tile `sub`, chunks in the order c ^ sub; head_dim 64: chunks
-      // 4 sub .. 4 sub + 3 of the one sub-tile
-      const int chunk = a.D == 128 ? (c ^ sub) : (4 * sub + c);
-      if (a.D == 128 || c < 4) {
-        const uint4 q = *reinterpret_cast<const uint4*>(stage + (a.D == 128 ? sub * kVSubBytes : 0) + row * 128 +
-                                                        ((chunk ^ (row & 7)) << 4));
-        float f[8];
-        if (a.bf16) Vec16<__nv_bfloat16>::widen(q, f);
-        else Vec16<__half>::widen(q, f);
+      for (int c = 0; c < 8; ++c) {
+        // head_dim 128: lane `sub` takes sub-tile `sub`, chunks in the order c ^ sub; head_dim 64: chunks
+        // 4 sub .. 4 sub + 3 of the one sub-tile
+        const int chunk = a.D == 128 ? (c ^ sub) : (4 * sub + c);
+        if (a.D == 128 || c < 4) {
+          const uint4 q = *reinterpret_cast<const uint4*>(stage + (a.D == 128 ? sub * kVSubBytes : 0) + row * 128 +
+                                                          ((chunk ^ (row & 7)) << 4));
+          float f[8];
+          if (a.bf16) Vec16<__nv_bfloat16>::widen(q, f);
+          else Vec16<__half>::widen(q, f);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc[e & 3] = fmaf(f[e], f[e], acc[e & 3]);
+          for (int e = 0; e < 8; ++e) acc[e & 3] = fmaf(f[e], f[e], acc[e & 3]);
+        }
       }
+      mbar_arrive(&bars->v_empty[vs]);
+      float sq = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+      sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+      const int j = cc.row0 + cc.t * kVRows + row;
+      if (sub == 0 && j < a.n) a.nu[(size_t)cc.bh * a.n + j] = sq;
     }
-    mbar_arrive(&bars->v_empty[vs]);
-    float sq = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-    sq += __shfl_xor_sync(0xffffffffu, sq, 1);
-    const int j = cc.row0 + cc.t * kVRows + row;
-    if (sub == 0 && j < a.n) a.nu[(size_t)cc.bh * a.n + j] = sq;
-    cv = v_advance(a, nr, cc);
+    ++cc.idx;
   }
+  if (leader) *(volatile int*)&sh->seg_done_v = 0x3fffffff;
 }
 
 // One k-step of a product.  The descriptors differ from their tile's base only in the address field
@@ -520,7 +610,7 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tm
   bool ok = true;
   const uint64_t fold_desc = umma_desc_ext(smem_u32(tiles + kOffExt + 2 * kExtBytes));
   const int nk = a.D / 16;
-  for_each_segment(a, [&](int pass, int run) {
+  for_each_segment(a, sh, [&](int pass, int run, int) {
     if (!ok) return;
     const Run rn = run_info(a, run);
     const int qb = sc & 1;
@@ -656,7 +746,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
   const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
   int tc = 0, p1c = 0;
   bool gone = false;   // a wait ran out: keep only the barriers
-  for_each_segment(a, [&](int pass, int run) {
+  for_each_segment(a, sh, [&](int pass, int run, int idx) {
     const Run rn = run_info(a, run);
     const UnitInfo u = unit_info(a, rn.unit);
     if (pass == 0) {
@@ -748,6 +838,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
         if (half == 0 && !gone && j < a.n) a.s_raw[(size_t)rn.unit * a.n + j] = sum + sh->p2_part[pair][buf][jl];
       }
     }
+    if (pair == 0 && half == 0 && s == 0) *(volatile int*)&sh->seg_done_soft = idx + 1;   // lets the scheduler publish on
   });
 }
 
@@ -781,16 +872,16 @@ __device__ __forceinline__ void write_extension(char* ext, int row, float off, f
   dst[1] = make_uint4(w0, w1, 0u, 0u);
 }
 
-// Merge group (two warps, 64 threads).  For every run of this CTA, in order and up to two runs ahead of
-// the MMA warp: thread `s` waits until the partials of rows 2s and 2s + 1 have arrived from all runs of the
+// Merge group (two warps, 64 threads).  For every pass-2 run the scheduler announces, in order and
+// ahead of the MMA warp: thread `s` waits until the partials of rows 2s and 2s + 1 have arrived from all runs of the
 // row block, merges them in run order into the rows' offsets and writes their offset extensions into
 // shared memory.
 __device__ void merge_group(const TcArgs& a, Shared* sh, char* tiles, int s) {
   Barriers* bars = &sh->bars;
-  const int G = (int)gridDim.x, first = (int)blockIdx.x;
-  const int nr = (a.n_runs - first + G - 1) / G;
-  for (int mc = 0; mc < nr; ++mc) {
-    const Run rn = run_info(a, first + mc * G);
+  for (int mc = 0;; ++mc) {
+    const int run = mrg_get(sh, mc, a.status);
+    if (run == kSegEnd) return;
+    const Run rn = run_info(a, run);
     const UnitInfo u = unit_info(a, rn.unit);
     const int slot = mc & 1;
     if (!mbar_wait(&bars->ext_empty[slot], ((mc >> 1) & 1) ^ 1, a.status)) return;
@@ -837,6 +928,7 @@ __device__ void merge_group(const TcArgs& a, Shared* sh, char* tiles, int s) {
     write_extension(ext, r1, M1 + log2f(Z1) + a.log2G, sh->c[obs_row(a, u, r1 < u.rows ? r1 : 0)], a.bf16, r1 < u.rows);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads it through the async proxy
     mbar_arrive(&bars->ext_full[slot]);
+    if (s == 0) *(volatile int*)&sh->mrg_done = mc + 1;
   }
 }
 
@@ -890,6 +982,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
       mbar_init(&bars->acc_full[s], 1);
       mbar_init(&bars->acc_empty[s], 256);
     }
+    sh->seg_pub = 0; sh->seg_done_soft = 0; sh->seg_done_v = a.prior ? 0 : 0x3fffffff;
+    sh->mrg_pub = 0; sh->mrg_done = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // all 512 TMEM columns: four 128-column accumulators
@@ -957,7 +1051,7 @@ bool make_map(CUtensorMap* m, const void* base, int bf16, int d, long long token
 bool score_tc_available() { return encode_fn() != nullptr; }
 
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
-                             float2* partial_ws, int* status, cudaStream_t st) {
+                             float2* partial_ws, int* counters, int* status, cudaStream_t st) {
   static int n_sm = 0;
   static bool configured = false;
   if (!configured) {
@@ -978,22 +1072,13 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   a.rpu = (pl.n_blk + a.CH - 1) / a.CH;
   a.n_runs = units * a.rpu;
   const int grid = a.n_runs < n_sm ? a.n_runs : n_sm;
-  // Pass 2 of a run follows its pass 1 by `lead` steps.  At least as many as the steps a row block's runs
-  // are spread over, so that a wait only depends on earlier work; beyond that, as many as keep about
-  // 40 MB of keys between the passes (L2 still holds that next to the rest of the traffic).
-  const long long step_bytes = (long long)grid * a.CH * kKeyTile * pl.d * pl.es;
-  long long lead = (40LL << 20) / (step_bytes > 0 ? step_bytes : 1);
-  if (lead > 3) lead = 3;
-  const long long spread = (a.rpu - 1 + grid - 1) / grid;
-  if (lead < spread) lead = spread;
-  if (lead < 1) lead = 1;
-  a.lead = (int)lead;
   a.bf16 = pl.dtype == AHAKV_BF16;
   a.prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0 && v != nullptr && nu != nullptr;
   a.log2G = log2f((float)pl.G);
   for (int i = 0; i < kMaxRows; ++i) a.c[i] = pl.rows.c[i];
   for (int t = 0; t < 128; ++t) a.cs[t] = pl.r <= 128 ? pl.rows.c[t % pl.r] : 0.f;
   a.partial = reinterpret_cast<float*>(partial_ws); a.s_raw = s_raw; a.nu = nu;
+  a.ctr = counters;
   a.status = status;
 
   CUtensorMap qmap, kmap, vmap;
