@@ -121,9 +121,11 @@ static ahakv_status check_ws(const Plan& pl, void* ws, size_t ws_bytes) {
 
 template <typename T> static T* at(void* ws, size_t off) { return reinterpret_cast<T*>((char*)ws + off); }
 
-// Queues the scoring kernels; the refined score lands in `score`.
+// Queues the scoring kernels; the refined score lands in `score`.  With `kept_idx` the selection is queued
+// too, in the same launch as the refinement when a head's scores fit in one CTA's registers.
 static ahakv_status queue_score(const Plan& pl, const void* q, const void* k, const void* v,
-                                const float* score_prev, float* score, void* ws, cudaStream_t st, int prof) {
+                                const float* score_prev, float* score, int32_t* kept_idx, void* ws, cudaStream_t st,
+                                int prof) {
   ahakv_status rc = cuda_ok(cudaMemsetAsync(at<char>(ws, pl.off_status), 0, pl.off_sraw - pl.off_status, st));
   if (rc) return rc;
   profile_mark(prof, 0, st);
@@ -144,8 +146,14 @@ static ahakv_status queue_score(const Plan& pl, const void* q, const void* k, co
     if (rc) return rc;
   }
   profile_mark(prof, 2, st);
+  if (kept_idx && refine_select_fits(pl)) {
+    rc = launch_refine_select(pl, s_raw, nu, score_prev, score, kept_idx, st);
+    profile_mark(prof, 3, st);
+    return rc;
+  }
   rc = launch_refine(pl, s_raw, nu, score_prev, score, st);
   profile_mark(prof, 3, st);
+  if (rc == AHAKV_OK && kept_idx) rc = launch_select(pl, score, kept_idx, st);
   return rc;
 }
 
@@ -179,7 +187,7 @@ ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k
     return AHAKV_ERR_INVALID_ARG;
   if ((rc = check_ws(pl, ws, ws_bytes))) return rc;
   const int prof = profile_begin_call((cudaStream_t)stream);
-  rc = queue_score(pl, q_obs, k, v, score_prev, score, ws, (cudaStream_t)stream, prof);
+  rc = queue_score(pl, q_obs, k, v, score_prev, score, nullptr, ws, (cudaStream_t)stream, prof);
   profile_mark(prof, 4, (cudaStream_t)stream);   // no selection or compaction in this call
   profile_mark(prof, 5, (cudaStream_t)stream);
   return rc;
@@ -222,8 +230,7 @@ ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k
   cudaStream_t st = (cudaStream_t)stream;
   float* score = at<float>(ws, pl.off_score);
   const int prof = profile_begin_call(st);
-  if ((rc = queue_score(pl, q_obs, k, v, score_prev, score, ws, st, prof))) return rc;
-  if ((rc = launch_select(pl, score, kept_idx, st))) return rc;
+  if ((rc = queue_score(pl, q_obs, k, v, score_prev, score, kept_idx, ws, st, prof))) return rc;
   profile_mark(prof, 4, st);
   rc = launch_compact(pl, k, v, score_out ? score : nullptr, kept_idx, k_out, v_out, score_out, st);
   profile_mark(prof, 5, st);

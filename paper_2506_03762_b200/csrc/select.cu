@@ -50,8 +50,8 @@ __global__ void __launch_bounds__(kThreads) refine_kernel(const float* __restric
   for (int j = threadIdx.x; j < n; j += kThreads) {
     float s = s_raw[(size_t)unit * slots * n + j];
     for (int t = 1; t < slots; ++t) s += s_raw[((size_t)unit * slots + t) * n + j];
-    if (prior) s = (pooled(nu_u, j, n, half, inv_full) / gmax) * s;
-    if (prev) s += prev[(size_t)unit * n + j];
+    if (prior) s = __fmul_rn(__fdiv_rn(pooled(nu_u, j, n, half, inv_full), gmax), s);
+    if (prev) s = __fadd_rn(s, prev[(size_t)unit * n + j]);
     score[(size_t)unit * n + j] = s;
   }
 }
@@ -62,10 +62,38 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// The digit at which the count of keys, taken from the largest digit down, reaches `need`: a suffix scan of
+// the 256-bin histogram by 256 threads.  Writes the extended prefix and how many keys of that digit are still
+// needed; ends with a barrier.
+__device__ __forceinline__ void find_digit(const unsigned* hist, unsigned need, unsigned prefix, int shift,
+                                           unsigned* out_prefix, unsigned* out_need, unsigned* warp_tot) {
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  unsigned h = 0, inc = 0;
+  if (t < 256) {
+    h = hist[255 - t];                         // thread t looks at digit 255 - t
+    inc = h;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned x = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += x;
+    }
+    if (lane == 31) warp_tot[warp] = inc;
+  }
+  __syncthreads();
+  if (t < 256) {
+    for (int w = 0; w < warp; ++w) inc += warp_tot[w];
+    if (inc >= need && inc - h < need) {       // exactly one digit crosses
+      *out_prefix = prefix | ((unsigned)(255 - t) << shift);
+      *out_need = need - (inc - h);
+    }
+  }
+  __syncthreads();
+}
+
 __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restrict__ score, int32_t* __restrict__ kept,
                                                           const Plan pl) {
   __shared__ unsigned hist[256];
-  __shared__ unsigned sh_prefix, sh_need;
+  __shared__ unsigned sh_prefix, sh_need, scan_tot[8];
   __shared__ int warp_gt[kWarps], warp_eq[kWarps];
   __shared__ int run_gt, run_eq;
   const int unit = blockIdx.x, n = pl.n;
@@ -91,17 +119,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restric
       if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      unsigned acc = 0;
-      int dgt = 255;
-      for (; dgt > 0; --dgt) {
-        if (acc + hist[dgt] >= need) break;
-        acc += hist[dgt];
-      }
-      sh_prefix = prefix | ((unsigned)dgt << shift);
-      sh_need = need - acc;                 // taken from the bucket `dgt`
-    }
-    __syncthreads();
+    find_digit(hist, need, prefix, shift, &sh_prefix, &sh_need, scan_tot);
     prefix = sh_prefix;
     need = sh_need;
     __syncthreads();
@@ -137,6 +155,160 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restric
   }
 }
 
+// Refinement and selection of one (sequence, KV head) in one CTA, for n <= 32 * kThreads.  Thread t owns
+// tokens t, t + kThreads, t + 2 kThreads, ... (coalesced) and keeps their refined scores in registers from the
+// first load to the last store: the value prior is applied once, and the four radix passes and the ordered
+// emission never go back to memory.  Same arithmetic, in the same order, as refine_kernel and select_kernel.
+constexpr int kPer = 32;
+
+__global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float* __restrict__ s_raw,
+                                                                    const float* __restrict__ nu,
+                                                                    const float* __restrict__ prev,
+                                                                    float* __restrict__ score, int32_t* __restrict__ kept,
+                                                                    const Plan pl, const int slots) {
+  __shared__ float red[kWarps];
+  __shared__ unsigned hist[256];
+  __shared__ unsigned sh_prefix, sh_need, scan_tot[8];
+  __shared__ int2 cnt[kPer * kWarps];      // kept-candidate counts (greater, equal) per 32-token group, in token order
+  const int unit = blockIdx.x, n = pl.n, half = pl.pool / 2;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const bool prior = nu != nullptr;
+  const float inv_full = (pl.flags & AHAKV_FLAG_POOL_ZERO_PAD) ? 1.f / (float)pl.pool : 0.f;
+  const float* nu_u = prior ? nu + (size_t)unit * n : nullptr;
+
+  uint32_t key[kPer];                                       // first the bits of gamma, then the score's order key
+  float gmax = 1.f;
+  if (prior) {
+    // the head's value norms go to shared memory in one coalesced sweep; the mean filter reads them there
+    extern __shared__ float nu_s[];
+    {
+      float v[kPer];
+#pragma unroll
+      for (int e = 0; e < kPer; ++e) {
+        const int j = e * kThreads + threadIdx.x;
+        v[e] = j < n ? nu_u[j] : 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < kPer; ++e) {
+        const int j = e * kThreads + threadIdx.x;
+        if (j < n) nu_s[j] = v[e];
+      }
+    }
+    __syncthreads();
+    float m = 0.f;
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) {
+      const int j = e * kThreads + threadIdx.x;
+      const float g = j < n ? pooled(nu_s, j, n, half, inv_full) : 0.f;
+      key[e] = __float_as_uint(g);
+      m = fmaxf(m, g);
+    }
+    gmax = block_max(m, red);
+  }
+#pragma unroll
+  for (int e0 = 0; e0 < kPer; e0 += 8) {                   // eight tokens' loads in flight at a time
+    float sr[8], pv[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int j = (e0 + e) * kThreads + threadIdx.x;
+      sr[e] = 0.f; pv[e] = 0.f;
+      if (j < n) {
+        sr[e] = s_raw[(size_t)unit * slots * n + j];
+        for (int t = 1; t < slots; ++t) sr[e] += s_raw[((size_t)unit * slots + t) * n + j];
+        if (prev) pv[e] = prev[(size_t)unit * n + j];
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int j = (e0 + e) * kThreads + threadIdx.x;
+      const float g = prior ? __uint_as_float(key[e0 + e]) : 0.f;
+      key[e0 + e] = 0u;
+      if (j < n) {
+        float s = sr[e];
+        if (prior) s = __fmul_rn(__fdiv_rn(g, gmax), s);
+        if (prev) s = __fadd_rn(s, pv[e]);
+        score[(size_t)unit * n + j] = s;
+        key[e0 + e] = order_key(s);
+      }
+    }
+  }
+
+  int32_t* out = kept + (size_t)unit * pl.n_keep;
+  if (n <= pl.Bud) {                       // nothing to evict
+#pragma unroll
+    for (int e = 0; e < kPer; ++e)
+      if (e * kThreads + threadIdx.x < n) out[e * kThreads + threadIdx.x] = e * kThreads + threadIdx.x;
+    return;
+  }
+  const int n_cand = n - pl.Br, Bs = pl.Bs;
+  for (int t = threadIdx.x; t < pl.Br; t += kThreads) out[Bs + t] = n_cand + t;   // recent window
+  if (Bs == 0) return;
+
+  // ---- radix select on the keys in registers: key of the Bs-th largest candidate ----
+  unsigned prefix = 0, need = (unsigned)Bs;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    const unsigned mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
+    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < kPer; ++e) {
+      const bool in = e * kThreads + (int)threadIdx.x < n_cand && (key[e] & mask) == prefix;
+      const unsigned digit = (key[e] >> shift) & 255u;
+      // one atomic per distinct digit of the warp
+      const unsigned live = __ballot_sync(0xffffffffu, in);
+      if (in) {
+        const unsigned same = __match_any_sync(live, digit);
+        if (lane == __ffs(same) - 1) atomicAdd(&hist[digit], (unsigned)__popc(same));
+      }
+    }
+    __syncthreads();
+    find_digit(hist, need, prefix, shift, &sh_prefix, &sh_need, scan_tot);
+    prefix = sh_prefix;
+    need = sh_need;
+    __syncthreads();
+  }
+  const unsigned thr = prefix;
+  const int need_eq = (int)need;
+
+  // ---- ordered emission: counts per 32-token group, one scan over the groups, then the writes ----
+#pragma unroll
+  for (int e = 0; e < kPer; ++e) {
+    const bool c = e * kThreads + (int)threadIdx.x < n_cand;
+    const unsigned bg = __ballot_sync(0xffffffffu, c && key[e] > thr), be = __ballot_sync(0xffffffffu, c && key[e] == thr);
+    if (lane == 0) cnt[e * kWarps + warp] = make_int2(__popc(bg), __popc(be));
+  }
+  __syncthreads();
+  {
+    // exclusive scan of the 1024 group counts, in place: thread t owns group t (kPer * kWarps == kThreads)
+    const int2 v = cnt[threadIdx.x];
+    int2 inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int x = __shfl_up_sync(0xffffffffu, inc.x, o), y = __shfl_up_sync(0xffffffffu, inc.y, o);
+      if (lane >= o) { inc.x += x; inc.y += y; }
+    }
+    __shared__ int2 warp_tot[kWarps];
+    if (lane == 31) warp_tot[warp] = inc;
+    __syncthreads();
+    int2 base = make_int2(0, 0);
+    for (int w = 0; w < warp; ++w) { base.x += warp_tot[w].x; base.y += warp_tot[w].y; }
+    cnt[threadIdx.x] = make_int2(base.x + inc.x - v.x, base.y + inc.y - v.y);
+    __syncthreads();
+  }
+  const unsigned below = (1u << lane) - 1u;
+#pragma unroll
+  for (int e = 0; e < kPer; ++e) {
+    const int j = e * kThreads + threadIdx.x;
+    const bool c = j < n_cand;
+    const bool gt = c && key[e] > thr, eq = c && key[e] == thr;
+    const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+    const int2 b0 = cnt[e * kWarps + warp];
+    const int gt_before = b0.x + __popc(bg & below), eq_before = b0.y + __popc(be & below);
+    if (gt || (eq && eq_before < need_eq)) out[gt_before + min(eq_before, need_eq)] = j;
+  }
+}
+
 }  // namespace
 
 ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
@@ -148,6 +320,26 @@ ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, 
 
 ahakv_status launch_select(const Plan& pl, const float* score, int32_t* kept_idx, cudaStream_t st) {
   select_kernel<<<pl.B * pl.Hkv, kThreads, 0, st>>>(score, kept_idx, pl);
+  count_launch();
+  return cuda_ok(cudaGetLastError());
+}
+
+
+// Both steps in one launch when a head's scores fit in the registers of one CTA; false if they do not.
+bool refine_select_fits(const Plan& pl) { return pl.n <= kPer * kThreads; }
+
+ahakv_status launch_refine_select(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
+                                  float* score, int32_t* kept_idx, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    if (cudaFuncSetAttribute(refine_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kPer * kThreads * (int)sizeof(float)) != cudaSuccess)
+      return AHAKV_ERR_CUDA;
+    configured = true;
+  }
+  const size_t smem = nu ? (size_t)pl.n * sizeof(float) : 0;
+  refine_select_kernel<<<pl.B * pl.Hkv, kThreads, smem, st>>>(s_raw, nu, score_prev, score, kept_idx, pl,
+                                                              pl.use_tc ? pl.n_rb : 1);
   count_launch();
   return cuda_ok(cudaGetLastError());
 }
