@@ -591,6 +591,16 @@ __device__ void v_group(const TcArgs& a, Shared* sh, char* tiles) {
 
 // One k-step of a product.  The descriptors differ from their tile's base only in the address field
 // (bits 0-13, in 16-byte units), so a k-step costs one add per operand.
+// Low word of umma_desc(): the address field and the (unused) leading byte offset.  The high word is the
+// same for every 128-byte-swizzled K-major tile.
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3ffff) >> 4) | (1u << 16); }
+constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+
 template <int ACC>
 __device__ __forceinline__ void umma_step(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
   const uint32_t accumulate = ACC;
@@ -632,12 +642,14 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tm
       if (!(ok = mbar_wait(&bars->k_full[stage], ph, a.status))) return;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 128);
-      const uint32_t q_addr = smem_u32(tiles + kOffQ + qb * kQBytes), k_addr = smem_u32(tiles + kOffK + stage * kKStageBytes);
+      const uint32_t q_lo = umma_desc_lo(smem_u32(tiles + kOffQ + qb * kQBytes));
+      const uint32_t k_lo = umma_desc_lo(smem_u32(tiles + kOffK + stage * kKStageBytes));
 #pragma unroll
       for (int kk = 0; kk < 8; ++kk) {
-        // k-step kk reads 32 bytes at offset (kk & 3) * 32 of sub-tile kk >> 2
-        const uint32_t off = (uint32_t)((kk >> 2) * kSubTileBytes + (kk & 3) * 32);
-        const uint64_t qd = umma_desc(q_addr + off), kd = umma_desc(k_addr + off);
+        // k-step kk reads 32 bytes at offset (kk & 3) * 32 of sub-tile kk >> 2: the address field moves by
+        // that many 16-byte units (tiles are 1024-byte aligned, so nothing carries out of the field)
+        const uint32_t off = (uint32_t)(((kk >> 2) * kSubTileBytes + (kk & 3) * 32) >> 4);
+        const uint64_t qd = desc64(q_lo + off, kDescHi), kd = desc64(k_lo + off, kDescHi);
         if (kk < nk) {
           if (kk == 0) umma_step<0>(d_tmem, pass == 0 ? qd : kd, pass == 0 ? kd : qd, idesc);
           else umma_step<1>(d_tmem, pass == 0 ? qd : kd, pass == 0 ? kd : qd, idesc);
