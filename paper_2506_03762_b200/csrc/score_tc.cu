@@ -154,13 +154,17 @@ __device__ __forceinline__ bool mbar_try(void* bar, int parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false (and records the timeout) if the phase did not complete in time.
+// Bounded wait.  Returns false (and records the timeout) if the phase did not complete in time.  The
+// clock is slow to read, so it is looked at only after many failed tries (each of which already sleeps in
+// hardware for a while).
 __device__ __forceinline__ bool mbar_wait(void* bar, int parity, int* status) {
-  if (mbar_try(bar, parity)) return true;
+#pragma unroll 1
+  for (int t = 0; t < 256; ++t)
+    if (mbar_try(bar, parity)) return true;
   const long long t0 = now_ns();
   for (;;) {
 #pragma unroll 1
-    for (int t = 0; t < 64; ++t)
+    for (int t = 0; t < 256; ++t)
       if (mbar_try(bar, parity)) return true;
     if (now_ns() - t0 > kWaitLimitNs) {
       atomicExch(status, (int)AHAKV_ERR_TIMEOUT);
@@ -338,11 +342,13 @@ __device__ __forceinline__ int seg_peek(Shared* sh, int idx) {
 __device__ __forceinline__ int seg_get(Shared* sh, int idx, int* status) {
   int e = seg_peek(sh, idx);
   if (e != -2) return e;
-  const long long t0 = now_ns();
-  for (;;) {
+  long long t0 = -1;
+  for (int spins = 0;; ++spins) {
     __nanosleep(64);
     if ((e = seg_peek(sh, idx)) != -2) return e;
-    if (now_ns() - t0 > kWaitLimitNs) {
+    if ((spins & 255) != 255) continue;                   // the clock is slow to read
+    if (t0 < 0) t0 = now_ns();
+    else if (now_ns() - t0 > kWaitLimitNs) {
       atomicExch(status, (int)AHAKV_ERR_TIMEOUT);
       return kSegEnd;
     }
@@ -469,6 +475,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
 
   Scheduler sched = {0, 0, -1, true, true, false};
   long long idle_since = -1;
+  int idle_spins = 0;
   while (k_state != 3 || v_state != 3) {
     bool progress = false;
     // a new round whenever the K stream is about to run dry
@@ -533,7 +540,8 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
     }
     if (progress) {
       idle_since = -1;
-    } else {
+      idle_spins = 0;
+    } else if ((++idle_spins & 1023) == 0) {               // the clock is slow to read: look at it rarely
       const long long now = now_ns();
       if (idle_since < 0) idle_since = now;
       else if (now - idle_since > kWaitLimitNs) {
