@@ -624,7 +624,7 @@ __device__ __forceinline__ void umma_step(uint32_t tmem_d, uint64_t adesc, uint6
 // Pass 1: D[rows x keys] = Q K^T.  Pass 2: D[keys x rows] = K Q^T - off / c.
 __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tmem_base) {
   Barriers* bars = &sh->bars;
-  int tc = 0, sc = 0, pc = 0;
+  int tc = 0, sc = 0, pc = 0, used0 = 0, used1 = 0;   // used: tiles handed to each softmax pair so far
   bool ok = true;
   const uint64_t fold_desc = umma_desc_ext(smem_u32(tiles + kOffExt + 2 * kExtBytes));
   const int nk = a.D / 16;
@@ -645,7 +645,10 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tm
     }
     for (int t = 0; t < rn.cnt; ++t, ++tc) {
       const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
-      const int acc = (tc & 1) * 2 + ((tc >> 1) & 1), aph = (tc >> 2) & 1;
+      // tile t of a run goes to softmax pair t & 1, whatever came before: the split of a run over the pairs,
+      // and with it the rounding of its statistics, must not depend on the CTA's history
+      const int pr = t & 1, used = pr ? used1++ : used0++;
+      const int acc = pr * 2 + (used & 1), aph = (used >> 1) & 1;
       if (!(ok = mbar_wait(&bars->acc_empty[acc], aph ^ 1, a.status))) return;
       if (!(ok = mbar_wait(&bars->k_full[stage], ph, a.status))) return;
       tc_fence_after();
@@ -753,8 +756,8 @@ __device__ __forceinline__ float column_sum_fast(const TcArgs& a, uint32_t taddr
   return (z0 + z1) + (z2 + z3);
 }
 
-// Softmax warps: sixteen warps in two pairs of 4-warp groups.  Tiles alternate between the pairs (tile
-// counter parity); within a pair the two groups split the accumulator's columns in halves.
+// Softmax warps: sixteen warps in two pairs of 4-warp groups.  The tiles of a run alternate between the pairs
+// (tile t of the run goes to pair t & 1); within a pair the two groups split the accumulator's columns in halves.
 //   pass 1: thread `s` of a group owns stacked row s over its 64 key columns; at the end of the run the
 //           four groups' (shift, sum) pairs meet in shared memory and one group publishes the row's
 //           partial, log2 of the sum, with one 4-byte store.
@@ -764,7 +767,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
   Barriers* bars = &sh->bars;
   const int s = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
   const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-  int tc = 0, p1c = 0;
+  int tc = 0, p1c = 0, mine = 0;   // mine: tiles this pair has been handed so far
   bool gone = false;   // a wait ran out: keep only the barriers
   for_each_segment(a, sh, [&](int pass, int run, int idx) {
     const Run rn = run_info(a, run);
@@ -775,8 +778,10 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
       const int last = a.n - a.r + i;                       // last visible key of this row
       float M = -INFINITY, Z = 0.f;
       for (int t = 0; t < rn.cnt; ++t, ++tc) {
-        if ((tc & 1) != pair || gone) continue;
-        const int acc = pair * 2 + ((tc >> 1) & 1), aph = (tc >> 2) & 1;
+        if ((t & 1) != pair) continue;
+        const int used = mine++;
+        if (gone) continue;
+        const int acc = pair * 2 + (used & 1), aph = (used >> 1) & 1;
         if (!mbar_wait(&bars->acc_full[acc], aph, a.status)) { gone = true; continue; }
         tc_fence_after();
         const int j0 = (rn.blk0 + t) * kKeyTile + 64 * half;
@@ -822,8 +827,9 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
       const float* cs = sh->cs2[u.rb & 1];
       const int* last_key = sh->vis_off[u.rb & 1];
       for (int t = 0; t < rn.cnt; ++t, ++tc) {
-        if ((tc & 1) != pair) continue;
-        const int buf = (tc >> 1) & 1, acc = pair * 2 + buf, aph = (tc >> 2) & 1;
+        if ((t & 1) != pair) continue;
+        const int used = mine++;
+        const int buf = used & 1, acc = pair * 2 + buf, aph = (used >> 1) & 1;
         const int j0 = (rn.blk0 + t) * kKeyTile, j = j0 + jl;
         float sum = 0.f;
         if (!gone && !mbar_wait(&bars->acc_full[acc], aph, a.status)) gone = true;
@@ -1087,7 +1093,8 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   a.n = pl.n; a.r = pl.r; a.G = pl.G; a.Hkv = pl.Hkv; a.n_rb = pl.n_rb; a.hb = pl.heads_per_rb;
   a.n_blk = pl.n_blk; a.D = pl.d;
   const long long tiles = (long long)units * pl.n_blk;
-  const long long ch = tiles / ((long long)n_sm * 8);
+  // runs of up to 8 tiles, but at least two runs per SM so that every SM has work on small problems
+  const long long ch = tiles / ((long long)n_sm * 2);
   a.CH = ch < 1 ? 1 : (ch > 8 ? 8 : (int)ch);
   a.rpu = (pl.n_blk + a.CH - 1) / a.CH;
   a.n_runs = units * a.rpu;

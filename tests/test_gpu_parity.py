@@ -112,6 +112,8 @@ EDGE_CASES = [
     (3, 6, 2, 64, 260, 40, 10, 77, ab.F32, dict(n_total=100000)),         # G = 3: rows do not fill a block
     (1, 1, 1, 128, 64, 64, 8, 32, ab.F16, {}),                             # r == n: every row is causal
     (1, 1, 1, 64, 1, 1, 1, 1, ab.F32, {}),                                 # a single token
+    (1, 2, 1, 64, 33500, 16, 32, 600, ab.F16, {}),                        # more scores per head than one CTA's registers hold
+    (1, 2, 2, 128, 128 * 23 + 5, 40, 16, 300, ab.BF16, {}),                # odd run lengths, three row-block-sized heads
 ]
 
 
@@ -151,15 +153,21 @@ def test_strided_cache_layout():
         assert torch.equal(a, b)
 
 
-def test_runs_are_bitwise_reproducible():
-    w = synth.WORKLOADS["llama2_7b_4k"]
+@pytest.mark.parametrize("name,over", [("llama2_7b_4k", {}), ("decode_round", dict(batch=8)),
+                                       ("llama3_8b_gqa_16k", dict(batch=1, n_ctx=128 * 37 + 11))])
+def test_runs_are_bitwise_reproducible(name, over):
+    """Runs are handed to the CTAs in whatever order they come free; the result must not depend on it."""
+    w = synth.WORKLOADS[name].scaled(**over)
     p = parity.params_of(w)
     q, k, v = synth.make_layer(w, device=DEV)
-    first = parity.run_evict(p, q, k, v)
+    prev = synth.make_score_prev(w, device=DEV, new_rows=w.obs_window) if w.n_total is not None else None
+    first = parity.run_evict(p, q, k, v, prev)
+    score = parity.run_score(p, q, k, v, prev)
     for _ in range(3):
-        again = parity.run_evict(p, q, k, v)
+        again = parity.run_evict(p, q, k, v, prev)
         for a, b in zip(first, again):
             assert torch.equal(a, b)
+        assert torch.equal(parity.run_score(p, q, k, v, prev), score)
 
 
 # ---- the separate entry points ----------------------------------------------------------------------------
