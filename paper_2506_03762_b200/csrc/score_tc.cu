@@ -917,15 +917,23 @@ __device__ void merge_group(const TcArgs& a, Shared* sh, char* tiles, int s) {
       float2 e[16];
       const long long tstart = now_ns();
       for (;;) {
-        bool all = true;
+        int missing = -1;
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
           e[t] = t0 + t < a.rpu ? ld_partial2(&p[(size_t)(t0 + t) * 64]) : make_float2(-INFINITY, -INFINITY);
-          all = all && (e[t].x == e[t].x) && (e[t].y == e[t].y);   // NaN: not published yet
+          if (!(e[t].x == e[t].x) || !(e[t].y == e[t].y)) missing = t;   // NaN: not published yet
         }
-        if (all) break;
-        __nanosleep(300);
-        if (now_ns() - tstart > kWaitLimitNs) {
+        if (missing < 0) break;
+        // wait for that one partial alone before looking at the batch again: sixteen loads per thread and try
+        // from every CTA that is early would keep L2 busy for nothing
+        bool timed_out = false;
+        for (;;) {
+          __nanosleep(400);
+          const float2 x = ld_partial2(&p[(size_t)(t0 + missing) * 64]);
+          if (x.x == x.x && x.y == x.y) break;
+          if (now_ns() - tstart > kWaitLimitNs) { timed_out = true; break; }
+        }
+        if (timed_out) {
           // nothing more is delivered; the MMA warp's own wait then runs out too
           atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
           return;

@@ -28,8 +28,16 @@ __device__ __forceinline__ float block_max(float x, float* red) {
 
 __device__ __forceinline__ float pooled(const float* __restrict__ nu, int j, int n, int half, float inv_full) {
   const int lo = max(j - half, 0), hi = min(j + half, n - 1);
-  float s = 0.f;
-  for (int t = lo; t <= hi; ++t) s += nu[t];
+  float s;
+  if (hi - lo == 6) {
+    // the usual width (7) away from the ends: seven independent loads, added in the order of the loop below
+    const float a0 = nu[lo], a1 = nu[lo + 1], a2 = nu[lo + 2], a3 = nu[lo + 3], a4 = nu[lo + 4], a5 = nu[lo + 5],
+                a6 = nu[lo + 6];
+    s = (((((a0 + a1) + a2) + a3) + a4) + a5) + a6;
+  } else {
+    s = 0.f;
+    for (int t = lo; t <= hi; ++t) s += nu[t];
+  }
   return inv_full > 0.f ? s * inv_full : s / (float)(hi - lo + 1);
 }
 
