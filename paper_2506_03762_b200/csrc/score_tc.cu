@@ -1086,16 +1086,19 @@ bool score_tc_available() { return encode_fn() != nullptr; }
 
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
                              float2* partial_ws, int* counters, int* status, cudaStream_t st) {
-  static int n_sm = 0;
-  static bool configured = false;
-  if (!configured) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+  // once per device: its SM count, and leave to use more than 48 KB of dynamic shared memory
+  constexpr int kMaxDevices = 64;
+  static int sm_count[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AHAKV_ERR_CUDA;
+  if (sm_count[dev] == 0) {
+    int count = 0;
+    if (cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || count <= 0 ||
         cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
       return AHAKV_ERR_CUDA;
-    configured = true;
+    sm_count[dev] = count;
   }
+  const int n_sm = sm_count[dev];
   const int units = pl.B * pl.Hkv * pl.n_rb;
   TcArgs a;
   a.n = pl.n; a.r = pl.r; a.G = pl.G; a.Hkv = pl.Hkv; a.n_rb = pl.n_rb; a.hb = pl.heads_per_rb;

@@ -163,12 +163,15 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restric
   }
 }
 
-// Refinement and selection of one (sequence, KV head) in one CTA, for n <= 32 * kThreads.  Thread t owns
+// Refinement and selection of one (sequence, KV head) in one CTA, for n <= kPer * kThreads.  Thread t owns
 // tokens t, t + kThreads, t + 2 kThreads, ... (coalesced) and keeps their refined scores in registers from the
 // first load to the last store: the value prior is applied once, and the four radix passes and the ordered
 // emission never go back to memory.  Same arithmetic, in the same order, as refine_kernel and select_kernel.
-constexpr int kPer = 32;
+// kPer is the number of tokens a thread owns (every loop below is unrolled over it, so a short context is not
+// made to pay for the longest one).
+constexpr int kPerMax = 32;
 
+template <int kPer>
 __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float* __restrict__ s_raw,
                                                                     const float* __restrict__ nu,
                                                                     const float* __restrict__ prev,
@@ -213,11 +216,12 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
     }
     gmax = block_max(m, red);
   }
+  constexpr int kBatch = kPer < 8 ? kPer : 8;
 #pragma unroll
-  for (int e0 = 0; e0 < kPer; e0 += 8) {                   // eight tokens' loads in flight at a time
-    float sr[8], pv[8];
+  for (int e0 = 0; e0 < kPer; e0 += kBatch) {              // eight tokens' loads in flight at a time
+    float sr[kBatch], pv[kBatch];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
+    for (int e = 0; e < kBatch; ++e) {
       const int j = (e0 + e) * kThreads + threadIdx.x;
       sr[e] = 0.f; pv[e] = 0.f;
       if (j < n) {
@@ -227,7 +231,7 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
       }
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
+    for (int e = 0; e < kBatch; ++e) {
       const int j = (e0 + e) * kThreads + threadIdx.x;
       const float g = prior ? __uint_as_float(key[e0 + e]) : 0.f;
       key[e0 + e] = 0u;
@@ -288,8 +292,9 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
   }
   __syncthreads();
   {
-    // exclusive scan of the 1024 group counts, in place: thread t owns group t (kPer * kWarps == kThreads)
-    const int2 v = cnt[threadIdx.x];
+    // exclusive scan of the kPer * kWarps (<= kThreads) group counts, in place: thread t owns group t
+    const bool mine = (int)threadIdx.x < kPer * kWarps;
+    const int2 v = mine ? cnt[threadIdx.x] : make_int2(0, 0);
     int2 inc = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -301,7 +306,7 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
     __syncthreads();
     int2 base = make_int2(0, 0);
     for (int w = 0; w < warp; ++w) { base.x += warp_tot[w].x; base.y += warp_tot[w].y; }
-    cnt[threadIdx.x] = make_int2(base.x + inc.x - v.x, base.y + inc.y - v.y);
+    if (mine) cnt[threadIdx.x] = make_int2(base.x + inc.x - v.x, base.y + inc.y - v.y);
     __syncthreads();
   }
   const unsigned below = (1u << lane) - 1u;
@@ -334,22 +339,40 @@ ahakv_status launch_select(const Plan& pl, const float* score, int32_t* kept_idx
 
 
 // Both steps in one launch when a head's scores fit in the registers of one CTA; false if they do not.
-bool refine_select_fits(const Plan& pl) { return pl.n <= kPer * kThreads; }
+bool refine_select_fits(const Plan& pl) { return pl.n <= kPerMax * kThreads; }
+
+namespace {
+template <int kPer>
+ahakv_status launch_refine_select_as(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
+                                     float* score, int32_t* kept_idx, cudaStream_t st) {
+  // more than 48 KB of dynamic shared memory has to be asked for once per device
+  constexpr int kMaxDevices = 64;
+  static bool configured[kMaxDevices] = {};
+  const size_t smem = nu ? (size_t)pl.n * sizeof(float) : 0;
+  if (smem > 48 * 1024) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AHAKV_ERR_CUDA;
+    if (!configured[dev]) {
+      if (cudaFuncSetAttribute(refine_select_kernel<kPer>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               kPer * kThreads * (int)sizeof(float)) != cudaSuccess)
+        return AHAKV_ERR_CUDA;
+      configured[dev] = true;
+    }
+  }
+  refine_select_kernel<kPer><<<pl.B * pl.Hkv, kThreads, smem, st>>>(s_raw, nu, score_prev, score, kept_idx, pl,
+                                                                    pl.use_tc ? pl.n_rb : 1);
+  count_launch();
+  return cuda_ok(cudaGetLastError());
+}
+}  // namespace
 
 ahakv_status launch_refine_select(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
                                   float* score, int32_t* kept_idx, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
-    if (cudaFuncSetAttribute(refine_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kPer * kThreads * (int)sizeof(float)) != cudaSuccess)
-      return AHAKV_ERR_CUDA;
-    configured = true;
-  }
-  const size_t smem = nu ? (size_t)pl.n * sizeof(float) : 0;
-  refine_select_kernel<<<pl.B * pl.Hkv, kThreads, smem, st>>>(s_raw, nu, score_prev, score, kept_idx, pl,
-                                                              pl.use_tc ? pl.n_rb : 1);
-  count_launch();
-  return cuda_ok(cudaGetLastError());
+  const int per = (pl.n + kThreads - 1) / kThreads;          // tokens a thread owns
+  if (per <= 4) return launch_refine_select_as<4>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+  if (per <= 8) return launch_refine_select_as<8>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+  if (per <= 16) return launch_refine_select_as<16>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+  return launch_refine_select_as<kPerMax>(pl, s_raw, nu, score_prev, score, kept_idx, st);
 }
 
 }  // namespace ahakv
