@@ -114,6 +114,9 @@ EDGE_CASES = [
     (1, 1, 1, 64, 1, 1, 1, 1, ab.F32, {}),                                 # a single token
     (1, 2, 1, 64, 33500, 16, 32, 600, ab.F16, {}),                        # more scores per head than one CTA's registers hold
     (1, 2, 2, 128, 128 * 23 + 5, 40, 16, 300, ab.BF16, {}),                # odd run lengths, three row-block-sized heads
+    (1, 2, 1, 64, 4097, 16, 32, 500, ab.F16, {}),                          # fused refine+select: 8 tokens a thread, barely
+    (1, 1, 1, 64, 8192, 16, 32, 900, ab.BF16, {}),                         # ... 8 tokens a thread, exactly
+    (1, 1, 1, 64, 8193, 16, 32, 900, ab.F16, {}),                          # ... 16 tokens a thread, barely
 ]
 
 
