@@ -89,6 +89,34 @@ def test_decode_rounds_chain_through_the_compacted_cache():
     parity.check_units(p2, q2, k2, v2, [(0, 0), (1, 5)], score_prev=prev2)
 
 
+def test_per_step_generation_update_chains_to_the_batched_round():
+    """Algorithm 1's generation phase one token at a time: F_t = SGsoftmax(A_t) + F_{t-1}, each step a call with
+    one observation row, the grown cache and the carried score (0 for the new row).  After T steps the score
+    must equal one call with T observation rows over the final cache, and the oracle's."""
+    B, Hq, Hkv, d, n0, T, N0 = 2, 8, 2, 128, 1500, 8, 20000
+    g = torch.Generator(device="cpu").manual_seed(77)
+    k_all = torch.randn((B, Hkv, n0 + T, d), generator=g).to(torch.bfloat16).to(DEV)
+    q_all = torch.randn((B, Hq, T, d), generator=g).to(torch.bfloat16).to(DEV)
+    v_all = torch.randn((B, Hkv, n0 + T, d), generator=g).to(torch.bfloat16).to(DEV)    # not read: no value prior here
+    f = (torch.rand((B, Hkv, n0), generator=g) * 0.01).to(DEV)
+    f0 = f.clone()
+    for t in range(T):
+        n = n0 + t + 1
+        p = ab.Params(B, Hq, Hkv, d, n, 1, 16, 512, dtype=ab.BF16, n_total=N0 + t + 1, flags=0)
+        prev = torch.cat([f, torch.zeros((B, Hkv, 1), device=DEV)], 2).contiguous()
+        f = parity.run_score(p, q_all[:, :, t:t + 1].contiguous(), k_all[:, :, :n].contiguous(),
+                             v_all[:, :, :n].contiguous(), prev)
+    n = n0 + T
+    pT = ab.Params(B, Hq, Hkv, d, n, T, 16, 512, dtype=ab.BF16, n_total=N0 + T, flags=0)
+    prevT = torch.cat([f0, torch.zeros((B, Hkv, T), device=DEV)], 2).contiguous()
+    batched = parity.run_score(pT, q_all, k_all, v_all, prevT)
+    parity.assert_scores_close(pT, f.cpu().numpy(), batched.cpu().numpy(), "chained vs batched")
+    for b, h in [(0, 0), (1, 1)]:
+        op, qn, kn, vn, sp = parity.unit_inputs(pT, q_all, k_all, v_all, b, h, prevT)
+        ref = orc.evict(op, qn, kn, vn, sp)
+        parity.assert_scores_close(pT, f[b, h].cpu().numpy(), ref["score"][0, 0], "chained vs oracle")
+
+
 # ---- small shapes: tiles, ragged tails, degenerate cases ---------------------------------------------
 
 EDGE_CASES = [
