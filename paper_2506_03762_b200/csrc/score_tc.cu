@@ -189,20 +189,8 @@ __device__ __forceinline__ void tc_commit(void* bar) {
                : "memory");
 }
 
-// Shared-memory operand descriptor: K-major tile of 128-byte rows, 128-byte swizzle, 8-row groups
-// 1024 bytes apart, descriptor version 1 (sm_100).
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr & 0x3ffff) >> 4);          // start address
-  d |= (uint64_t)1 << 16;                               // leading byte offset (unused with swizzle)
-  d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset
-  d |= (uint64_t)1 << 46;                               // version
-  d |= (uint64_t)2 << 61;                               // SWIZZLE_128B
-  return d;
-}
-
-// The same for a K-major tile of 32-byte rows (16 elements, one k-step), 32-byte swizzle, 8-row groups
-// 256 bytes apart.
+// Shared-memory operand descriptor (fields as described at umma_desc_lo below) of a K-major tile of 32-byte
+// rows (16 elements, one k-step), 32-byte swizzle, 8-row groups 256 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc_ext(uint32_t smem_addr) {
   uint64_t d = 0;
   d |= (uint64_t)((smem_addr & 0x3ffff) >> 4);
@@ -597,10 +585,11 @@ __device__ void v_group(const TcArgs& a, Shared* sh, char* tiles) {
   if (leader) *(volatile int*)&sh->seg_done_v = 0x3fffffff;
 }
 
-// One k-step of a product.  The descriptors differ from their tile's base only in the address field
-// (bits 0-13, in 16-byte units), so a k-step costs one add per operand.
-// Low word of umma_desc(): the address field and the (unused) leading byte offset.  The high word is the
-// same for every 128-byte-swizzled K-major tile.
+// Shared-memory operand descriptor of a K-major tile of 128-byte rows with 128-byte swizzle: start address
+// (bits 0-13, in 16-byte units), leading byte offset (bits 16-29, unused with swizzle, set to 1), stride byte
+// offset between 8-row groups (bits 32-45: 1024 bytes), descriptor version 1 of sm_100 (bit 46), swizzle mode
+// (bits 61-63: 2 = 128 bytes).  Only the address field differs between the k-steps of a tile, so the low word
+// is made per tile and a k-step costs one add per operand; the high word is a constant.
 __device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3ffff) >> 4) | (1u << 16); }
 constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
