@@ -112,7 +112,7 @@ struct Shared {
   float cs2[2][128];            // c per stacked row, by row block parity (r > 128 has two kinds of block)
   int vis_off[2][128];          // per stacked row: n - r + its observation row = the last key it may see
   float2 p1_part[2][3][128];    // pass 1: statistics of the three groups that do not publish
-  float p2_part[2][2][128];     // pass 2: partial column sums of the second half of the rows, per pair
+  float p2_part[2][3][128];     // pass 2: partial column sums of the three groups that do not store
 };
 
 constexpr int kQBytes = 2 * kSubTileBytes;              // D <= 128
@@ -124,8 +124,8 @@ constexpr int kOffK = kOffQ + 2 * kQBytes;
 constexpr int kOffV = kOffK + kKStages * kKStageBytes;
 constexpr int kOffExt = kOffV + kVStages * kVStageBytes;        // two extensions, then the constant tile
 constexpr int kSmemTiles = kOffExt + 3 * kExtBytes;      // 204 KiB
-constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 12288 /*barriers, constants, exchange*/;
-static_assert(sizeof(Shared) <= 12288, "Shared outgrew its reservation");
+constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 13312 /*barriers, constants, exchange*/;
+static_assert(sizeof(Shared) <= 13312, "Shared outgrew its reservation");
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -613,7 +613,7 @@ __device__ __forceinline__ void umma_step(uint32_t tmem_d, uint64_t adesc, uint6
 // Pass 1: D[rows x keys] = Q K^T.  Pass 2: D[keys x rows] = K Q^T - off / c.
 __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tmem_base) {
   Barriers* bars = &sh->bars;
-  int tc = 0, sc = 0, pc = 0, used0 = 0, used1 = 0;   // used: tiles handed to each softmax pair so far
+  int tc = 0, sc = 0, pc = 0;
   bool ok = true;
   const uint64_t fold_desc = umma_desc_ext(smem_u32(tiles + kOffExt + 2 * kExtBytes));
   const int nk = a.D / 16;
@@ -634,10 +634,7 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tm
     }
     for (int t = 0; t < rn.cnt; ++t, ++tc) {
       const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
-      // tile t of a run goes to softmax pair t & 1, whatever came before: the split of a run over the pairs,
-      // and with it the rounding of its statistics, must not depend on the CTA's history
-      const int pr = t & 1, used = pr ? used1++ : used0++;
-      const int acc = pr * 2 + (used & 1), aph = (used >> 1) & 1;
+      const int acc = tc & 3, aph = (tc >> 2) & 1;      // the four accumulators in turn
       if (!(ok = mbar_wait(&bars->acc_empty[acc], aph ^ 1, a.status))) return;
       if (!(ok = mbar_wait(&bars->k_full[stage], ph, a.status))) return;
       tc_fence_after();
@@ -723,40 +720,40 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
   }
 }
 
-// Sixty-four stacked rows of a key's column, rows [64 HALF, 64 HALF + 64): adds 2^{c D} of each.  The
-// column indices are compile-time constants, so every c comes straight from the kernel's parameter
-// bank as an operand of the multiply.
-template <int HALF>
-__device__ __forceinline__ float column_sum_fast(const TcArgs& a, uint32_t taddr) {
+// Thirty-two stacked rows of a key's column, rows [32 Q, 32 Q + 32): adds 2^{c D} of each.  The column
+// indices are compile-time constants, so every c comes straight from the kernel's parameter bank as an operand
+// of the multiply.  The accumulator goes back to the MMA thread as soon as the values are in registers.
+template <int Q>
+__device__ __forceinline__ float column_sum_fast(const TcArgs& a, uint32_t taddr, void* acc_empty) {
+  uint32_t r[32];
+  tmem_ld32_issue(taddr + 32 * Q, r);
+  tmem_ld_wait(r);
+  tc_fence_before();
+  mbar_arrive(acc_empty);
   float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    uint32_t r[16];
-    tmem_ld16_issue(taddr + 64 * HALF + 16 * q, r);
-    tmem_ld_wait16(r);
-#pragma unroll
-    for (int t = 0; t < 16; t += 4) {
-      z0 += fast_exp2(__uint_as_float(r[t]) * a.cs[64 * HALF + 16 * q + t]);
-      z1 += fast_exp2(__uint_as_float(r[t + 1]) * a.cs[64 * HALF + 16 * q + t + 1]);
-      z2 += fast_exp2(__uint_as_float(r[t + 2]) * a.cs[64 * HALF + 16 * q + t + 2]);
-      z3 += fast_exp2(__uint_as_float(r[t + 3]) * a.cs[64 * HALF + 16 * q + t + 3]);
-    }
+  for (int t = 0; t < 32; t += 4) {
+    z0 += fast_exp2(__uint_as_float(r[t]) * a.cs[32 * Q + t]);
+    z1 += fast_exp2(__uint_as_float(r[t + 1]) * a.cs[32 * Q + t + 1]);
+    z2 += fast_exp2(__uint_as_float(r[t + 2]) * a.cs[32 * Q + t + 2]);
+    z3 += fast_exp2(__uint_as_float(r[t + 3]) * a.cs[32 * Q + t + 3]);
   }
   return (z0 + z1) + (z2 + z3);
 }
 
-// Softmax warps: sixteen warps in two pairs of 4-warp groups.  The tiles of a run alternate between the pairs
-// (tile t of the run goes to pair t & 1); within a pair the two groups split the accumulator's columns in halves.
-//   pass 1: thread `s` of a group owns stacked row s over its 64 key columns; at the end of the run the
+// Softmax warps: sixteen warps in four 4-warp groups, all of them on every tile (the four accumulators are used
+// in turn); group g takes a quarter of the accumulator's columns, reads it with one load and hands the
+// accumulator back before its arithmetic.  Which thread adds what does not depend on the schedule.
+//   pass 1: thread `s` of a group owns stacked row s over its 32 key columns; at the end of the run the
 //           four groups' (shift, sum) pairs meet in shared memory and one group publishes the row's
 //           partial, log2 of the sum, with one 4-byte store.
-//   pass 2: thread `jl` owns key j0 + jl over its half of the stacked rows; the second group of the pair
-//           hands its partial sum over through shared memory, the first adds the two and stores.
-__device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int pair, int half) {
+//   pass 2: thread `jl` owns key j0 + jl over its quarter of the stacked rows; three groups hand their partial
+//           sums over through shared memory, the first adds the four in a fixed order and stores.
+__device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int g) {
   Barriers* bars = &sh->bars;
   const int s = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
   const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
-  int tc = 0, p1c = 0, mine = 0;   // mine: tiles this pair has been handed so far
+  int tc = 0, p1c = 0;   // tiles and pass-1 runs seen so far
   bool gone = false;   // a wait ran out: keep only the barriers
   for_each_segment(a, sh, [&](int pass, int run, int idx) {
     const Run rn = run_info(a, run);
@@ -767,34 +764,26 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
       const int last = a.n - a.r + i;                       // last visible key of this row
       float M = -INFINITY, Z = 0.f;
       for (int t = 0; t < rn.cnt; ++t, ++tc) {
-        if ((t & 1) != pair) continue;
-        const int used = mine++;
         if (gone) continue;
-        const int acc = pair * 2 + (used & 1), aph = (used >> 1) & 1;
+        const int acc = tc & 3, aph = (tc >> 2) & 1;
         if (!mbar_wait(&bars->acc_full[acc], aph, a.status)) { gone = true; continue; }
         tc_fence_after();
-        const int j0 = (rn.blk0 + t) * kKeyTile + 64 * half;
+        const int j0 = (rn.blk0 + t) * kKeyTile + 32 * g;
         const bool full = (rn.blk0 + t) * kKeyTile + kKeyTile - 1 <= a.n - a.r;   // no key of the tile is masked
-        const uint32_t taddr = lane_base + (uint32_t)(acc * 128 + 64 * half);
         uint32_t ra[32];
-        // One chunk at a time: load, wait, fold.  The other warps of the scheduler fill the load latency;
-        // keeping a second load in flight costs registers and ties the exponentials to its completion.
-        tmem_ld32_issue(taddr, ra);
-        tmem_ld_wait(ra);
-        fold_chunk(ra, full, j0, last, c, M, Z);
-        tmem_ld32_issue(taddr + 32, ra);
+        tmem_ld32_issue(lane_base + (uint32_t)(acc * 128 + 32 * g), ra);
         tmem_ld_wait(ra);
         tc_fence_before();
         mbar_arrive(&bars->acc_empty[acc]);                  // the accumulator is free for the next product
-        fold_chunk(ra, full, j0 + 32, last, c, M, Z);
+        fold_chunk(ra, full, j0, last, c, M, Z);
       }
       // All sixteen warps meet here once per run, also after a wait has run out, so that nobody is left
       // at the barrier.  Two slots: the others can be at most one run ahead of the publishing group's read.
-      const int slot = p1c & 1, who = pair * 2 + half;
+      const int slot = p1c & 1;
       ++p1c;
-      if (who != 0) sh->p1_part[slot][who - 1][s] = make_float2(M, Z);
+      if (g != 0) sh->p1_part[slot][g - 1][s] = make_float2(M, Z);
       group_sync(5, 512);
-      if (who == 0 && !gone) {
+      if (g == 0 && !gone) {
         float m = M;
 #pragma unroll
         for (int w = 0; w < 3; ++w) m = fmaxf(m, sh->p1_part[slot][w][s].x);
@@ -810,15 +799,13 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
       }
     } else {
       const int jl = s;
-      const int split = ((u.npad / 16 + 1) / 2) * 16;
-      const int c_lo = half ? split : 0, c_hi = half ? u.npad : split;   // this group's accumulator columns
+      const int k16 = u.npad / 16;
+      const int c_lo = (k16 * g / 4) * 16, c_hi = (k16 * (g + 1) / 4) * 16;   // this group's accumulator columns
       const bool fast = a.r <= 128 && u.rows == 128;
       const float* cs = sh->cs2[u.rb & 1];
       const int* last_key = sh->vis_off[u.rb & 1];
       for (int t = 0; t < rn.cnt; ++t, ++tc) {
-        if ((t & 1) != pair) continue;
-        const int used = mine++;
-        const int buf = used & 1, acc = pair * 2 + buf, aph = (used >> 1) & 1;
+        const int buf = tc & 1, acc = tc & 3, aph = (tc >> 2) & 1;
         const int j0 = (rn.blk0 + t) * kKeyTile, j = j0 + jl;
         float sum = 0.f;
         if (!gone && !mbar_wait(&bars->acc_full[acc], aph, a.status)) gone = true;
@@ -827,7 +814,9 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
           const bool full = j0 + kKeyTile - 1 <= a.n - a.r;
           const uint32_t taddr = lane_base + (uint32_t)(acc * 128);
           if (full && fast) {
-            sum = half ? column_sum_fast<1>(a, taddr) : column_sum_fast<0>(a, taddr);
+            void* ae = &bars->acc_empty[acc];
+            sum = g == 0 ? column_sum_fast<0>(a, taddr, ae) : g == 1 ? column_sum_fast<1>(a, taddr, ae)
+                : g == 2 ? column_sum_fast<2>(a, taddr, ae) : column_sum_fast<3>(a, taddr, ae);
           } else {
             // The product wrote exactly npad (a multiple of 16) columns; those past `rows` belong to no row.
 #pragma unroll 1
@@ -842,18 +831,19 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
                 if (vis) sum += fast_exp2(__uint_as_float(v[t2]) * cs[sr]);
               }
             }
+            tc_fence_before();
+            mbar_arrive(&bars->acc_empty[acc]);
           }
-          tc_fence_before();
-          mbar_arrive(&bars->acc_empty[acc]);
         }
-        // The two groups of the pair meet here once per tile, also after a wait has run out.  Two slots:
-        // the second group can be at most one tile ahead of the first group's read.
-        if (half == 1) sh->p2_part[pair][buf][jl] = sum;
-        group_sync(6 + pair, 256);
-        if (half == 0 && !gone && j < a.n) a.s_raw[(size_t)rn.unit * a.n + j] = sum + sh->p2_part[pair][buf][jl];
+        // The four groups meet here once per tile, also after a wait has run out.  Two slots: the others can be
+        // at most one tile ahead of the storing group's read.
+        if (g != 0) sh->p2_part[buf][g - 1][jl] = sum;
+        group_sync(6, 512);
+        if (g == 0 && !gone && j < a.n)
+          a.s_raw[(size_t)rn.unit * a.n + j] = ((sum + sh->p2_part[buf][0][jl]) + sh->p2_part[buf][1][jl]) + sh->p2_part[buf][2][jl];
       }
     }
-    if (pair == 0 && half == 0 && s == 0) *(volatile int*)&sh->seg_done_soft = idx + 1;   // lets the scheduler publish on
+    if (g == 0 && s == 0) *(volatile int*)&sh->seg_done_soft = idx + 1;   // lets the scheduler publish on
   });
 }
 
@@ -1003,7 +993,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
     }
     for (int s = 0; s < 4; ++s) {
       mbar_init(&bars->acc_full[s], 1);
-      mbar_init(&bars->acc_empty[s], 256);
+      mbar_init(&bars->acc_empty[s], 512);
     }
     sh->seg_pub = 0; sh->seg_done_soft = 0; sh->seg_done_v = a.prior ? 0 : 0x3fffffff;
     sh->mrg_pub = 0; sh->mrg_done = 0;
@@ -1025,7 +1015,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   } else if (warp < 4) {
     merge_group(a, sh, tiles, threadIdx.x & 63);
   } else if (warp < 20) {
-    softmax_group(a, sh, tmem_base, (warp - 4) >> 3, ((warp - 4) >> 2) & 1);
+    softmax_group(a, sh, tmem_base, (warp - 4) >> 2);
   } else {
     if (a.prior) v_group(a, sh, tiles);
   }
