@@ -671,6 +671,32 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tm
 // keeps every term finite, so the exponentials of a chunk are taken against the shift the row already
 // has, without waiting for the chunk's own maximum; only when that maximum outruns the shift by more
 // than the slack (or the row has no shift yet) is the chunk redone against a new shift.
+// Two FP32 operations an instruction (packed f32x2 on 64-bit register pairs): the softmax warps are bound by
+// the number of instructions they issue, and every pair of adds or multiply-adds done this way is one less.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 constexpr float kShiftSlack = 64.f;
 
 __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_first, int last, float c, float& M,
@@ -692,14 +718,19 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
   const float mx = fmaxf(mx0, mx1) * c;
   if (M > -INFINITY) {
     const float neg = -M;
-    float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+    const uint64_t c2 = pack2(c, c), neg2 = pack2(neg, neg);
+    uint64_t za = pack2(0.f, 0.f), zb = pack2(0.f, 0.f);
 #pragma unroll
     for (int t = 0; t < 32; t += 4) {
-      z0 += fast_exp2(fmaf(v[t], c, neg));
-      z1 += fast_exp2(fmaf(v[t + 1], c, neg));
-      z2 += fast_exp2(fmaf(v[t + 2], c, neg));
-      z3 += fast_exp2(fmaf(v[t + 3], c, neg));
+      float x0, x1, x2, x3;
+      unpack2(fma2(pack2(v[t], v[t + 1]), c2, neg2), x0, x1);
+      unpack2(fma2(pack2(v[t + 2], v[t + 3]), c2, neg2), x2, x3);
+      za = add2(za, pack2(fast_exp2(x0), fast_exp2(x1)));
+      zb = add2(zb, pack2(fast_exp2(x2), fast_exp2(x3)));
     }
+    float z0, z1, z2, z3;
+    unpack2(za, z0, z1);
+    unpack2(zb, z2, z3);
     if (mx <= M + kShiftSlack) {
       Z += (z0 + z1) + (z2 + z3);
       return;
@@ -707,14 +738,19 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
   }
   if (mx > -INFINITY) {                              // first visible keys of the row, or the shift fell behind
     const float neg = -mx;
-    float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+    const uint64_t c2 = pack2(c, c), neg2 = pack2(neg, neg);
+    uint64_t za = pack2(0.f, 0.f), zb = pack2(0.f, 0.f);
 #pragma unroll
     for (int t = 0; t < 32; t += 4) {
-      z0 += fast_exp2(fmaf(v[t], c, neg));
-      z1 += fast_exp2(fmaf(v[t + 1], c, neg));
-      z2 += fast_exp2(fmaf(v[t + 2], c, neg));
-      z3 += fast_exp2(fmaf(v[t + 3], c, neg));
+      float x0, x1, x2, x3;
+      unpack2(fma2(pack2(v[t], v[t + 1]), c2, neg2), x0, x1);
+      unpack2(fma2(pack2(v[t + 2], v[t + 3]), c2, neg2), x2, x3);
+      za = add2(za, pack2(fast_exp2(x0), fast_exp2(x1)));
+      zb = add2(zb, pack2(fast_exp2(x2), fast_exp2(x3)));
     }
+    float z0, z1, z2, z3;
+    unpack2(za, z0, z1);
+    unpack2(zb, z2, z3);
     Z = (M > -INFINITY ? Z * fast_exp2(M - mx) : 0.f) + ((z0 + z1) + (z2 + z3));
     M = mx;
   }
@@ -730,14 +766,17 @@ __device__ __forceinline__ float column_sum_fast(const TcArgs& a, uint32_t taddr
   tmem_ld_wait(r);
   tc_fence_before();
   mbar_arrive(acc_empty);
-  float z0 = 0.f, z1 = 0.f, z2 = 0.f, z3 = 0.f;
+  uint64_t za = pack2(0.f, 0.f), zb = pack2(0.f, 0.f);
 #pragma unroll
   for (int t = 0; t < 32; t += 4) {
-    z0 += fast_exp2(__uint_as_float(r[t]) * a.cs[32 * Q + t]);
-    z1 += fast_exp2(__uint_as_float(r[t + 1]) * a.cs[32 * Q + t + 1]);
-    z2 += fast_exp2(__uint_as_float(r[t + 2]) * a.cs[32 * Q + t + 2]);
-    z3 += fast_exp2(__uint_as_float(r[t + 3]) * a.cs[32 * Q + t + 3]);
+    za = add2(za, pack2(fast_exp2(__uint_as_float(r[t]) * a.cs[32 * Q + t]),
+                        fast_exp2(__uint_as_float(r[t + 1]) * a.cs[32 * Q + t + 1])));
+    zb = add2(zb, pack2(fast_exp2(__uint_as_float(r[t + 2]) * a.cs[32 * Q + t + 2]),
+                        fast_exp2(__uint_as_float(r[t + 3]) * a.cs[32 * Q + t + 3])));
   }
+  float z0, z1, z2, z3;
+  unpack2(za, z0, z1);
+  unpack2(zb, z2, z3);
   return (z0 + z1) + (z2 + z3);
 }
 
