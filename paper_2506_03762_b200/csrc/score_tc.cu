@@ -666,11 +666,6 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tm
   });
 }
 
-// One 32-key chunk of a row: fold it into the running pair (M, Z) with Z = sum of 2^{c w - M}.
-// M is a shift, not necessarily the maximum: any value within 2^kShiftSlack of the largest logit seen
-// keeps every term finite, so the exponentials of a chunk are taken against the shift the row already
-// has, without waiting for the chunk's own maximum; only when that maximum outruns the shift by more
-// than the slack (or the row has no shift yet) is the chunk redone against a new shift.
 // Two FP32 operations an instruction (packed f32x2 on 64-bit register pairs): the softmax warps are bound by
 // the number of instructions they issue, and every pair of adds or multiply-adds done this way is one less.
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
@@ -691,13 +686,15 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
 
+// One 32-key chunk of a row: fold it into the running pair (M, Z) with Z = sum of 2^{c w - M}.
+// M is a shift, not necessarily the maximum: any value within 2^kShiftSlack of the largest logit seen
+// keeps every term finite, so the exponentials of a chunk are taken against the shift the row already
+// has, and their sum tells whether that was sound: below 2^kShiftSlack, no term outran the shift by more
+// than the slack.  Only otherwise (or when the row has no shift yet) is the chunk's maximum looked for and
+// the chunk redone against it.
 constexpr float kShiftSlack = 64.f;
+constexpr float kAcceptBelow = 18446744073709551616.f;   // 2^kShiftSlack
 
 __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_first, int last, float c, float& M,
                                            float& Z) {
@@ -709,13 +706,6 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
     for (int t = 0; t < 32; ++t)
       if (j_first + t > last) v[t] = -INFINITY;
   }
-  float mx0 = fmaxf(v[0], v[1]), mx1 = fmaxf(v[2], v[3]);
-#pragma unroll
-  for (int t = 4; t < 32; t += 4) {
-    mx0 = fmaxf(mx0, fmaxf(v[t], v[t + 1]));
-    mx1 = fmaxf(mx1, fmaxf(v[t + 2], v[t + 3]));
-  }
-  const float mx = fmaxf(mx0, mx1) * c;
   if (M > -INFINITY) {
     const float neg = -M;
     const uint64_t c2 = pack2(c, c), neg2 = pack2(neg, neg);
@@ -731,11 +721,19 @@ __device__ __forceinline__ void fold_chunk(const uint32_t* r, bool full, int j_f
     float z0, z1, z2, z3;
     unpack2(za, z0, z1);
     unpack2(zb, z2, z3);
-    if (mx <= M + kShiftSlack) {
-      Z += (z0 + z1) + (z2 + z3);
+    const float z = (z0 + z1) + (z2 + z3);
+    if (z < kAcceptBelow) {                          // an overflow or a NaN fails this test too
+      Z += z;
       return;
     }
   }
+  float mx0 = fmaxf(v[0], v[1]), mx1 = fmaxf(v[2], v[3]);
+#pragma unroll
+  for (int t = 4; t < 32; t += 4) {
+    mx0 = fmaxf(mx0, fmaxf(v[t], v[t + 1]));
+    mx1 = fmaxf(mx1, fmaxf(v[t + 2], v[t + 3]));
+  }
+  const float mx = fmaxf(mx0, mx1) * c;
   if (mx > -INFINITY) {                              // first visible keys of the row, or the shift fell behind
     const float neg = -mx;
     const uint64_t c2 = pack2(c, c), neg2 = pack2(neg, neg);
