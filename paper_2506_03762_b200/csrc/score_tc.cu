@@ -1119,10 +1119,10 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   TcArgs a;
   a.n = pl.n; a.r = pl.r; a.G = pl.G; a.Hkv = pl.Hkv; a.n_rb = pl.n_rb; a.hb = pl.heads_per_rb;
   a.n_blk = pl.n_blk; a.D = pl.d;
-  const long long tiles = (long long)units * pl.n_blk;
-  // runs of up to 8 tiles, but at least two runs per SM so that every SM has work on small problems
-  const long long ch = tiles / ((long long)n_sm * 2);
-  a.CH = ch < 1 ? 1 : (ch > 8 ? 8 : (int)ch);
+  // Runs of 8 tiles; shorter ones (4, 2, 1) only as far as it takes to give three SMs in four a run.  Every run
+  // boundary drains the pipeline, which costs more than a few idle SMs on a small problem.
+  a.CH = 8;
+  while (a.CH > 1 && (long long)units * ((pl.n_blk + a.CH - 1) / a.CH) * 4 < (long long)n_sm * 3) a.CH >>= 1;
   a.rpu = (pl.n_blk + a.CH - 1) / a.CH;
   a.n_runs = units * a.rpu;
   const int grid = a.n_runs < n_sm ? a.n_runs : n_sm;
