@@ -270,8 +270,8 @@ __device__ __forceinline__ void st_partial(float* p, float v) {
 }
 
 // ---- work decomposition ----------------------------------------------------------------------------------
-// A run = up to CH consecutive key tiles of one row block.  Run `q` belongs to CTA q % gridDim.x; every role
-// of a CTA walks the same runs in the same order.
+// A run = up to CH consecutive key tiles of one row block.  Every role of a CTA walks the runs its scheduler
+// has taken, in the order of the CTA's segment ring.
 struct Run {
   int unit, rin, blk0, cnt;
 };
