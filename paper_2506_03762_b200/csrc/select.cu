@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restric
 // made to pay for the longest one).
 constexpr int kPerMax = 32;
 
-template <int kPer>
+template <int kPer, bool kPrev>
 __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float* __restrict__ s_raw,
                                                                     const float* __restrict__ nu,
                                                                     const float* __restrict__ prev,
@@ -216,7 +216,10 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
     }
     gmax = block_max(m, red);
   }
-  constexpr int kBatch = kPer < 8 ? kPer : 8;
+  // loads in flight at a time: without a carried score, and with fewer than 32 keys to hold, the registers allow
+  // twice as many
+  constexpr int kWide = (kPrev || kPer > 16) ? 8 : 16;
+  constexpr int kBatch = kPer < kWide ? kPer : kWide;
 #pragma unroll
   for (int e0 = 0; e0 < kPer; e0 += kBatch) {              // eight tokens' loads in flight at a time
     float sr[kBatch], pv[kBatch];
@@ -227,7 +230,7 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
       if (j < n) {
         sr[e] = s_raw[(size_t)unit * slots * n + j];
         for (int t = 1; t < slots; ++t) sr[e] += s_raw[((size_t)unit * slots + t) * n + j];
-        if (prev) pv[e] = prev[(size_t)unit * n + j];
+        if (kPrev) pv[e] = prev[(size_t)unit * n + j];
       }
     }
 #pragma unroll
@@ -238,7 +241,7 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
       if (j < n) {
         float s = sr[e];
         if (prior) s = __fmul_rn(__fdiv_rn(g, gmax), s);
-        if (prev) s = __fadd_rn(s, pv[e]);
+        if (kPrev) s = __fadd_rn(s, pv[e]);
         score[(size_t)unit * n + j] = s;
         key[e0 + e] = order_key(s);
       }
@@ -342,7 +345,7 @@ ahakv_status launch_select(const Plan& pl, const float* score, int32_t* kept_idx
 bool refine_select_fits(const Plan& pl) { return pl.n <= kPerMax * kThreads; }
 
 namespace {
-template <int kPer>
+template <int kPer, bool kPrev>
 ahakv_status launch_refine_select_as(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
                                      float* score, int32_t* kept_idx, cudaStream_t st) {
   // more than 48 KB of dynamic shared memory has to be asked for once per device
@@ -353,13 +356,13 @@ ahakv_status launch_refine_select_as(const Plan& pl, const float* s_raw, const f
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AHAKV_ERR_CUDA;
     if (!configured[dev]) {
-      if (cudaFuncSetAttribute(refine_select_kernel<kPer>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      if (cudaFuncSetAttribute(refine_select_kernel<kPer, kPrev>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                kPer * kThreads * (int)sizeof(float)) != cudaSuccess)
         return AHAKV_ERR_CUDA;
       configured[dev] = true;
     }
   }
-  refine_select_kernel<kPer><<<pl.B * pl.Hkv, kThreads, smem, st>>>(s_raw, nu, score_prev, score, kept_idx, pl,
+  refine_select_kernel<kPer, kPrev><<<pl.B * pl.Hkv, kThreads, smem, st>>>(s_raw, nu, score_prev, score, kept_idx, pl,
                                                                     pl.use_tc ? pl.n_rb : 1);
   count_launch();
   return cuda_ok(cudaGetLastError());
@@ -369,10 +372,16 @@ ahakv_status launch_refine_select_as(const Plan& pl, const float* s_raw, const f
 ahakv_status launch_refine_select(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
                                   float* score, int32_t* kept_idx, cudaStream_t st) {
   const int per = (pl.n + kThreads - 1) / kThreads;          // tokens a thread owns
-  if (per <= 4) return launch_refine_select_as<4>(pl, s_raw, nu, score_prev, score, kept_idx, st);
-  if (per <= 8) return launch_refine_select_as<8>(pl, s_raw, nu, score_prev, score, kept_idx, st);
-  if (per <= 16) return launch_refine_select_as<16>(pl, s_raw, nu, score_prev, score, kept_idx, st);
-  return launch_refine_select_as<kPerMax>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+  if (score_prev) {
+    if (per <= 4) return launch_refine_select_as<4, true>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+    if (per <= 8) return launch_refine_select_as<8, true>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+    if (per <= 16) return launch_refine_select_as<16, true>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+    return launch_refine_select_as<kPerMax, true>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+  }
+  if (per <= 4) return launch_refine_select_as<4, false>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+  if (per <= 8) return launch_refine_select_as<8, false>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+  if (per <= 16) return launch_refine_select_as<16, false>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+  return launch_refine_select_as<kPerMax, false>(pl, s_raw, nu, score_prev, score, kept_idx, st);
 }
 
 }  // namespace ahakv
