@@ -73,12 +73,14 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 // The digit at which the count of keys, taken from the largest digit down, reaches `need`: a suffix scan of
 // the 256-bin histogram by 256 threads.  Writes the extended prefix and how many keys of that digit are still
 // needed; ends with a barrier.
-__device__ __forceinline__ void find_digit(const unsigned* hist, unsigned need, unsigned prefix, int shift,
+template <int kCopies>
+__device__ __forceinline__ void find_digit(const unsigned (*hist)[256], unsigned need, unsigned prefix, int shift,
                                            unsigned* out_prefix, unsigned* out_need, unsigned* warp_tot) {
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   unsigned h = 0, inc = 0;
   if (t < 256) {
-    h = hist[255 - t];                         // thread t looks at digit 255 - t
+#pragma unroll
+    for (int c = 0; c < kCopies; ++c) h += hist[c][255 - t];   // thread t looks at digit 255 - t
     inc = h;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -100,7 +102,7 @@ __device__ __forceinline__ void find_digit(const unsigned* hist, unsigned need, 
 
 __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restrict__ score, int32_t* __restrict__ kept,
                                                           const Plan pl) {
-  __shared__ unsigned hist[256];
+  __shared__ unsigned hist[1][256];
   __shared__ unsigned sh_prefix, sh_need, scan_tot[8];
   __shared__ int warp_gt[kWarps], warp_eq[kWarps];
   __shared__ int run_gt, run_eq;
@@ -120,14 +122,14 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restric
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     const unsigned mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+    if (threadIdx.x < 256) hist[0][threadIdx.x] = 0;
     __syncthreads();
     for (int j = threadIdx.x; j < n_cand; j += kThreads) {
       const unsigned key = order_key(s[j]);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+      if ((key & mask) == prefix) atomicAdd(&hist[0][(key >> shift) & 255u], 1u);
     }
     __syncthreads();
-    find_digit(hist, need, prefix, shift, &sh_prefix, &sh_need, scan_tot);
+    find_digit<1>(hist, need, prefix, shift, &sh_prefix, &sh_need, scan_tot);
     prefix = sh_prefix;
     need = sh_need;
     __syncthreads();
@@ -170,6 +172,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restric
 // kPer is the number of tokens a thread owns (every loop below is unrolled over it, so a short context is not
 // made to pay for the longest one).
 constexpr int kPerMax = 32;
+constexpr int kHistCopies = 4;
 
 template <int kPer, bool kPrev>
 __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float* __restrict__ s_raw,
@@ -178,7 +181,9 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
                                                                     float* __restrict__ score, int32_t* __restrict__ kept,
                                                                     const Plan pl, const int slots) {
   __shared__ float red[kWarps];
-  __shared__ unsigned hist[256];
+  // four copies of the histogram, one per quarter of the warps: in the first passes nearly all keys of a head fall
+  // into one or two bins, and the atomics on one counter are served one after the other
+  __shared__ unsigned hist[kHistCopies][256];
   __shared__ unsigned sh_prefix, sh_need, scan_tot[8];
   __shared__ int2 cnt[kPer * kWarps];      // kept-candidate counts (greater, equal) per 32-token group, in token order
   const int unit = blockIdx.x, n = pl.n, half = pl.pool / 2;
@@ -264,7 +269,8 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     const unsigned mask = pass == 0 ? 0u : (0xffffffffu << (shift + 8));
-    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
+    static_assert(kHistCopies * 256 == kThreads, "one counter per thread to clear");
+    hist[threadIdx.x >> 8][threadIdx.x & 255] = 0;
     __syncthreads();
 #pragma unroll
     for (int e = 0; e < kPer; ++e) {
@@ -274,11 +280,11 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
       const unsigned live = __ballot_sync(0xffffffffu, in);
       if (in) {
         const unsigned same = __match_any_sync(live, digit);
-        if (lane == __ffs(same) - 1) atomicAdd(&hist[digit], (unsigned)__popc(same));
+        if (lane == __ffs(same) - 1) atomicAdd(&hist[warp & (kHistCopies - 1)][digit], (unsigned)__popc(same));
       }
     }
     __syncthreads();
-    find_digit(hist, need, prefix, shift, &sh_prefix, &sh_need, scan_tot);
+    find_digit<kHistCopies>(hist, need, prefix, shift, &sh_prefix, &sh_need, scan_tot);
     prefix = sh_prefix;
     need = sh_need;
     __syncthreads();
