@@ -37,7 +37,7 @@ extern "C" {
 typedef enum {
   AHAKV_OK = 0,
   AHAKV_ERR_INVALID_ARG = 1, /* a pointer, size, stride or parameter is wrong            */
-  AHAKV_ERR_UNSUPPORTED = 2, /* a legal request this build has no kernel for            */
+  AHAKV_ERR_UNSUPPORTED = 2, /* a legal request this library has no kernel for          */
   AHAKV_ERR_WORKSPACE = 3,   /* ws is null, misaligned or smaller than required          */
   AHAKV_ERR_CUDA = 4,        /* a CUDA runtime call or a launch failed                   */
   AHAKV_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (see last_device_status) */
