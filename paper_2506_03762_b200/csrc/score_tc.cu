@@ -990,6 +990,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   Shared* sh = reinterpret_cast<Shared*>(tiles + kSmemTiles);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {   // the copy engine's descriptors on their way while the CTA sets itself up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&qmap)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&kmap)) : "memory");
+    if (a.prior) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&vmap)) : "memory");
+  }
   for (int t = threadIdx.x; t < kMaxRows; t += kThreads) sh->c[t] = a.c[t];
   for (int t = threadIdx.x; t < 128; t += kThreads) {
     sh->cs2[0][t] = a.r <= 128 ? a.c[t % a.r] : a.c[t];
