@@ -330,10 +330,10 @@ def run_ours(args):
     dom = "score"
     achieved = stage_bytes[dom] / (stage_ms[dom] * 1e-3) / 1e9 if stage_ms[dom] > 0 else 0.0
     # DRAM bytes of one launch from the ncu capture summarised in profiles/score_tc_kernel_long32k_b2.txt:
-    # 1106.9 MB at batch 2, scaled by the units a launch of this run processes (traffic grows with them).
+    # 1108.4 MB at batch 2, scaled by the units a launch of this run processes (traffic grows with them).
     traffic = None
     if w.name == "long_32k" and w.value_prior:
-        traffic = 1106.9e6 * w.batch / 2
+        traffic = 1108.4e6 * w.batch / 2
     roofline = {"kernel": "score_tc_kernel (logits, SG-softmax, column sums, value norms)", "bound": "hbm",
                 "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
                 "peak_source": f"{pk['source']} (sustained copy)", "traffic": traffic,
