@@ -19,18 +19,23 @@ struct RowScale {
   float c[kMaxRows];
 };
 
-// Everything the host derives from ahakv_params once per call.
-struct Plan {
+// The sizes and strides of a call: the part of the plan that the small kernels take by value.
+struct Shape {
   int B, Hq, Hkv, G, d, n, r, Br, Bud, Bs, n_keep, dtype, es, pool;
   unsigned flags;
   long long n_total;
   int R;          // G * r
   int n_blk;      // ceil(n / kKeyTile)
+  long long qs[3], ks[3], vs[3];  // element strides: batch, head, token
+};
+
+// Everything the host derives from ahakv_params once per call.
+struct Plan : Shape {
   int n_rb;       // row blocks of 128 stacked rows (tensor-core path)
   int heads_per_rb;  // query heads per row block (tensor-core path)
   bool use_tc;    // tensor-core scoring path applies
-  long long qs[3], ks[3], vs[3];  // element strides: batch, head, token
   RowScale rows;
+  double lambda[kMaxRows];   // lambda_i itself, in double (the float32 path scales its logits in double)
   // workspace layout, byte offsets
   size_t off_status, off_sync, off_sraw, off_nu, off_partial, off_final, off_score, ws_total;
 };

@@ -72,17 +72,19 @@ ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
       !resolve_strides(p->v_stride, o.vs, o.Hkv, o.n, o.d, o.es))
     return AHAKV_ERR_INVALID_ARG;
 
-  for (int i = 0; i < kMaxRows; ++i) o.rows.c[i] = 0.f;
+  for (int i = 0; i < kMaxRows; ++i) { o.rows.c[i] = 0.f; o.lambda[i] = 0.0; }
   for (int i = 0; i < o.r; ++i) {
     double lam;
     if (p->scale_mode == AHAKV_SCALE_FIXED) lam = (double)p->scale;
     else if (p->scale_mode == AHAKV_SCALE_ADAPTIVE_ROW)
       lam = eq12((double)(p->n_total - p->obs_window + i + 1), (double)p->budget, p->head_dim);
     else lam = eq12((double)p->n_total, (double)p->budget, p->head_dim);
+    o.lambda[i] = lam;
     o.rows.c[i] = (float)(lam * 1.4426950408889634);
   }
 
-  // Tensor-core scoring: 16-bit inputs; query heads of a row block must form one TMA box.
+  // Tensor-core scoring: 16-bit inputs.  A row block stacks up to 128 / r query heads of one KV head (one TMA
+  // box); when G is not a multiple of that, the last block of each KV head simply holds fewer heads.
   o.heads_per_rb = 1; o.n_rb = 1; o.use_tc = false;
   if (o.es == 2 && o.n >= kKeyTile && (long long)o.B * o.Hkv * 2 * o.n_blk < (1LL << 30) && score_tc_available()) {
     if (o.r <= 128) {
@@ -90,7 +92,7 @@ ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
       if (hb > G) hb = G;
       o.heads_per_rb = hb;
       o.n_rb = (G + hb - 1) / hb;
-      o.use_tc = (G % hb == 0);
+      o.use_tc = true;
     } else {              // one query head split over two row blocks
       o.heads_per_rb = 1;
       o.n_rb = 2;

@@ -14,7 +14,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const char* __restric
                                                            const float* __restrict__ score,
                                                            const int32_t* __restrict__ kept, char* __restrict__ k_out,
                                                            char* __restrict__ v_out, float* __restrict__ score_out,
-                                                           const Plan pl) {
+                                                           const Shape pl) {
   const long long total = (long long)pl.B * pl.Hkv * pl.n_keep;
   const long long stride = (long long)gridDim.x * (kThreads / LANES);
   const int lane = threadIdx.x % LANES;

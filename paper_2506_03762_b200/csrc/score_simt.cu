@@ -7,6 +7,14 @@
 // tiles, and pass 2 recomputes the logits and adds the normalised weights of all
 // rows into the key's score (Eq. 1, 5, 9).  Every reduction has a fixed order,
 // so the scores are reproducible bit for bit.
+//
+// float32 inputs are held to 1e-5 on the scores, logits of hundreds included: an FP32
+// logit near 256 is only known to 3e-5, so for them the dot product, the scale and
+// the subtraction of the row's shift run in double (products of two floats are exact
+// there), and only the shifted exponent, a small number, goes back to FP32 for the
+// exponential.  16-bit inputs (1e-3) keep FP32 throughout.
+#include <type_traits>
+
 #include "ahakv_internal.cuh"
 
 namespace ahakv {
@@ -15,7 +23,7 @@ namespace {
 constexpr int kThreads = 128;
 
 template <typename T, int D>
-__device__ __forceinline__ void load_q_group(const T* __restrict__ q, const Plan& pl, int b, int h, float* qsm) {
+__device__ __forceinline__ void load_q_group(const T* __restrict__ q, const Shape& pl, int b, int h, float* qsm) {
   // qsm[s][c], s = g * r + i over the G query heads of KV head h
   constexpr int V = Vec16<T>::N;
   const int vec_per_row = D / V;
@@ -29,7 +37,7 @@ __device__ __forceinline__ void load_q_group(const T* __restrict__ q, const Plan
 }
 
 template <typename T, int D>
-__device__ __forceinline__ void load_key(const T* __restrict__ k, const Plan& pl, int b, int h, int j, float* kreg) {
+__device__ __forceinline__ void load_key(const T* __restrict__ k, const Shape& pl, int b, int h, int j, float* kreg) {
   constexpr int V = Vec16<T>::N;
   const T* row = k + (long long)b * pl.ks[0] + (long long)h * pl.ks[1] + (long long)j * pl.ks[2];
 #pragma unroll
@@ -39,16 +47,24 @@ __device__ __forceinline__ void load_key(const T* __restrict__ k, const Plan& pl
   }
 }
 
-template <int D>
-__device__ __forceinline__ float dot_row(const float* __restrict__ qrow, const float* kreg) {
-  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+// The accumulator type of the logits: double for float32 inputs, float for 16-bit ones.
+template <typename T> using Acc = typename std::conditional<std::is_same<T, float>::value, double, float>::type;
+
+// lambda_i log2(e) per observation row in the accumulator's type.
+template <typename A> struct RowScaleOf {
+  A c[kMaxRows];
+};
+
+template <int D, typename A>
+__device__ __forceinline__ A dot_row(const float* __restrict__ qrow, const float* kreg) {
+  A a0 = 0, a1 = 0, a2 = 0, a3 = 0;
 #pragma unroll
   for (int c = 0; c < D; c += 4) {
     const float4 qv = *reinterpret_cast<const float4*>(qrow + c);
-    a0 = fmaf(qv.x, kreg[c], a0);
-    a1 = fmaf(qv.y, kreg[c + 1], a1);
-    a2 = fmaf(qv.z, kreg[c + 2], a2);
-    a3 = fmaf(qv.w, kreg[c + 3], a3);
+    a0 = fma((A)qv.x, (A)kreg[c], a0);
+    a1 = fma((A)qv.y, (A)kreg[c + 1], a1);
+    a2 = fma((A)qv.z, (A)kreg[c + 2], a2);
+    a3 = fma((A)qv.w, (A)kreg[c + 3], a3);
   }
   return (a0 + a1) + (a2 + a3);
 }
@@ -56,7 +72,9 @@ __device__ __forceinline__ float dot_row(const float* __restrict__ qrow, const f
 // Pass 1: per (unit, key tile, stacked row) the pair (max of c*w, sum of 2^{c*w - max}).
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads) simt_row_stats(const T* __restrict__ q, const T* __restrict__ k,
-                                                           float2* __restrict__ partial, const Plan pl) {
+                                                           float2* __restrict__ partial, const Shape pl,
+                                                           const RowScaleOf<Acc<T>> cs) {
+  using A = Acc<T>;
   extern __shared__ __align__(16) float smem[];
   float* qsm = smem;                                            // [R][D]
   float2* wst = reinterpret_cast<float2*>(smem + pl.R * D);     // [4][R]
@@ -74,11 +92,11 @@ __global__ void __launch_bounds__(kThreads) simt_row_stats(const T* __restrict__
   for (int s = 0; s < pl.R; ++s) {
     const int i = s % pl.r;
     const bool vis = valid && j <= pl.n - pl.r + i;
-    const float x = vis ? dot_row<D>(qsm + s * D, kreg) * pl.rows.c[i] : -INFINITY;
-    float m = x;
+    const A x = vis ? dot_row<D, A>(qsm + s * D, kreg) * cs.c[i] : (A)-INFINITY;
+    float m = (float)x;                                         // the shift is an FP32 number on either path
 #pragma unroll
     for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float z = vis ? fast_exp2(x - m) : 0.f;
+    float z = vis ? fast_exp2((float)(x - (A)m)) : 0.f;
 #pragma unroll
     for (int o = 16; o; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
     if (lane == 0) wst[warp * pl.R + s] = make_float2(m, z);
@@ -100,7 +118,7 @@ __global__ void __launch_bounds__(kThreads) simt_row_stats(const T* __restrict__
 
 // Merge the tiles of one unit into (max, 1 / (G * sum)) per stacked row, so that
 // 2^{c w - max} times the second entry is the softmax weight divided by the group size.
-__global__ void simt_merge_stats(const float2* __restrict__ partial, float2* __restrict__ final_st, const Plan pl) {
+__global__ void simt_merge_stats(const float2* __restrict__ partial, float2* __restrict__ final_st, const Shape pl) {
   const int unit = blockIdx.x;
   for (int s = threadIdx.x; s < pl.R; s += blockDim.x) {
     const float2* p = partial + (size_t)unit * pl.n_blk * pl.R + s;
@@ -119,7 +137,9 @@ __global__ void simt_merge_stats(const float2* __restrict__ partial, float2* __r
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads) simt_column_sums(const T* __restrict__ q, const T* __restrict__ k,
                                                              const float2* __restrict__ final_st,
-                                                             float* __restrict__ s_raw, const Plan pl) {
+                                                             float* __restrict__ s_raw, const Shape pl,
+                                                             const RowScaleOf<Acc<T>> cs) {
+  using A = Acc<T>;
   extern __shared__ __align__(16) float smem[];
   float* qsm = smem;                                            // [R][D]
   float2* st = reinterpret_cast<float2*>(smem + pl.R * D);      // [R]
@@ -135,7 +155,7 @@ __global__ void __launch_bounds__(kThreads) simt_column_sums(const T* __restrict
   for (int s = 0; s < pl.R; ++s) {
     const int i = s % pl.r;
     if (j <= pl.n - pl.r + i)
-      acc = fmaf(fast_exp2(fmaf(dot_row<D>(qsm + s * D, kreg), pl.rows.c[i], -st[s].x)), st[s].y, acc);
+      acc = fmaf(fast_exp2((float)fma(dot_row<D, A>(qsm + s * D, kreg), cs.c[i], -(A)st[s].x)), st[s].y, acc);
   }
   s_raw[(size_t)unit * pl.n + j] = acc;
 }
@@ -143,16 +163,18 @@ __global__ void __launch_bounds__(kThreads) simt_column_sums(const T* __restrict
 template <typename T, int D>
 ahakv_status run(const Plan& pl, const void* q, const void* k, float* s_raw, float2* partial, float* final_off,
                  cudaStream_t st) {
+  RowScaleOf<Acc<T>> cs;
+  for (int i = 0; i < kMaxRows; ++i) cs.c[i] = i < pl.r ? (Acc<T>)(pl.lambda[i] * 1.4426950408889634) : (Acc<T>)0;
   const size_t smem1 = (size_t)pl.R * D * sizeof(float) + (size_t)(kThreads / 32) * pl.R * sizeof(float2);
   const size_t smem2 = (size_t)pl.R * D * sizeof(float) + (size_t)pl.R * sizeof(float2);
   if (cudaFuncSetAttribute(simt_row_stats<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||
       cudaFuncSetAttribute(simt_column_sums<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
     return AHAKV_ERR_CUDA;
   const dim3 grid(pl.n_blk, pl.B * pl.Hkv);
-  simt_row_stats<T, D><<<grid, kThreads, smem1, st>>>((const T*)q, (const T*)k, partial, pl);
+  simt_row_stats<T, D><<<grid, kThreads, smem1, st>>>((const T*)q, (const T*)k, partial, pl, cs);
   float2* final_st = reinterpret_cast<float2*>(final_off);
   simt_merge_stats<<<pl.B * pl.Hkv, 256, 0, st>>>(partial, final_st, pl);
-  simt_column_sums<T, D><<<grid, kThreads, smem2, st>>>((const T*)q, (const T*)k, final_st, s_raw, pl);
+  simt_column_sums<T, D><<<grid, kThreads, smem2, st>>>((const T*)q, (const T*)k, final_st, s_raw, pl, cs);
   count_launch(3);
   return cuda_ok(cudaGetLastError());
 }

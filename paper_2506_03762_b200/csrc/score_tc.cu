@@ -294,7 +294,10 @@ __device__ __forceinline__ UnitInfo unit_info(const TcArgs& a, int unit) {
   u.rb = unit % a.n_rb;
   u.b = u.bh / a.Hkv;
   u.h = u.bh % a.Hkv;
-  u.rows = a.r <= 128 ? a.hb * a.r : min(128, a.r - u.rb * 128);
+  // r <= 128: hb query heads a block, fewer in the last block of a KV head when hb does not divide G (the
+  // box still brings hb heads' rows; those past `rows` belong to another KV head or read as zeros, and no
+  // result depends on them)
+  u.rows = a.r <= 128 ? min(a.hb, a.G - u.rb * a.hb) * a.r : min(128, a.r - u.rb * 128);
   u.npad = (u.rows + 15) & ~15;
   return u;
 }

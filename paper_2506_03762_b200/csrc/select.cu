@@ -43,7 +43,7 @@ __device__ __forceinline__ float pooled(const float* __restrict__ nu, int j, int
 
 __global__ void __launch_bounds__(kThreads) refine_kernel(const float* __restrict__ s_raw, const float* __restrict__ nu,
                                                           const float* __restrict__ prev, float* __restrict__ score,
-                                                          const Plan pl, const int slots) {
+                                                          const Shape pl, const int slots) {
   __shared__ float red[kWarps];
   const int unit = blockIdx.x, n = pl.n, half = pl.pool / 2;
   const bool prior = nu != nullptr;
@@ -101,7 +101,7 @@ __device__ __forceinline__ void find_digit(const unsigned (*hist)[256], unsigned
 }
 
 __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restrict__ score, int32_t* __restrict__ kept,
-                                                          const Plan pl) {
+                                                          const Shape pl) {
   __shared__ unsigned hist[1][256];
   __shared__ unsigned sh_prefix, sh_need, scan_tot[8];
   __shared__ int warp_gt[kWarps], warp_eq[kWarps];
@@ -179,7 +179,7 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
                                                                     const float* __restrict__ nu,
                                                                     const float* __restrict__ prev,
                                                                     float* __restrict__ score, int32_t* __restrict__ kept,
-                                                                    const Plan pl, const int slots) {
+                                                                    const Shape pl, const int slots) {
   __shared__ float red[kWarps];
   // four copies of the histogram, one per quarter of the warps: in the first passes nearly all keys of a head fall
   // into one or two bins, and the atomics on one counter are served one after the other
@@ -354,11 +354,12 @@ namespace {
 template <int kPer, bool kPrev>
 ahakv_status launch_refine_select_as(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
                                      float* score, int32_t* kept_idx, cudaStream_t st) {
-  // more than 48 KB of dynamic shared memory has to be asked for once per device
+  // Static and dynamic shared memory together may pass 48 KB well before the dynamic part alone does, and
+  // beyond that the launch needs leave, asked for once per device: ask whenever the value norms are staged.
   constexpr int kMaxDevices = 64;
   static bool configured[kMaxDevices] = {};
   const size_t smem = nu ? (size_t)pl.n * sizeof(float) : 0;
-  if (smem > 48 * 1024) {
+  if (smem > 0) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AHAKV_ERR_CUDA;
     if (!configured[dev]) {

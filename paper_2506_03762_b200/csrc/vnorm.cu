@@ -16,7 +16,7 @@ __device__ __forceinline__ uint4 ld_stream(const void* p) {  // read once: do no
 }
 
 template <typename T, int LANES>
-__global__ void __launch_bounds__(kThreads) vnorm_kernel(const T* __restrict__ v, float* __restrict__ nu, const Plan pl) {
+__global__ void __launch_bounds__(kThreads) vnorm_kernel(const T* __restrict__ v, float* __restrict__ nu, const Shape pl) {
   constexpr int V = Vec16<T>::N;
   const long long total_rows = (long long)pl.B * pl.Hkv * pl.n;
   const long long groups = (long long)gridDim.x * (kThreads / LANES);

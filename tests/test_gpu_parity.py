@@ -145,6 +145,16 @@ EDGE_CASES = [
     (1, 2, 1, 64, 4097, 16, 32, 500, ab.F16, {}),                          # fused refine+select: 8 tokens a thread, barely
     (1, 1, 1, 64, 8192, 16, 32, 900, ab.BF16, {}),                         # ... 8 tokens a thread, exactly
     (1, 1, 1, 64, 8193, 16, 32, 900, ab.F16, {}),                          # ... 16 tokens a thread, barely
+    # value norms staged in 40 to 48 KB of dynamic shared memory next to the kernel's static arrays
+    (1, 1, 1, 64, 10133, 16, 32, 900, ab.F16, {}),
+    (1, 2, 1, 64, 11000, 16, 32, 900, ab.BF16, {}),
+    (1, 1, 1, 64, 12288, 16, 32, 900, ab.F16, {}),
+    (1, 1, 1, 64, 12288, 16, 32, 900, ab.BF16, dict(n_total=40000)),
+    # query heads that do not fill the last row block of their KV head
+    (1, 7, 1, 128, 1300, 32, 32, 300, ab.BF16, {}),                        # G = 7, r = 32: blocks of 4 + 3 heads
+    (2, 14, 2, 128, 1300, 32, 32, 300, ab.F16, {}),
+    (1, 5, 1, 64, 900, 48, 16, 200, ab.F16, {}),                           # G = 5, r = 48: blocks of 2 + 2 + 1 heads
+    (1, 3, 1, 128, 700, 80, 16, 200, ab.BF16, {}),                         # one head a block, 80 of 128 rows live
 ]
 
 
@@ -156,12 +166,25 @@ def test_edge_shapes(case):
     parity.check_units(p, q, k, v, parity.all_units(p))
 
 
+@pytest.mark.parametrize("Hq,r", [(7, 32), (5, 48), (28, 32)])
+def test_uneven_head_groups_take_the_tensor_core_path(Hq, r):
+    """Grouped queries whose heads do not fill the last 128-row block of their KV head (Qwen2-7B, the model of
+    the paper's Appendix E, has 28 query heads on 4 KV heads) must not fall back to the FP32-pipe kernels: an
+    eviction call is then three launches (scoring, refine+select, compact), not six."""
+    Hkv = 1 if Hq < 28 else 4
+    p = ab.Params(1, Hq, Hkv, 128, 2000, r, 32, 400, dtype=ab.BF16)
+    q, k, v = _rand_problem(1, Hq, Hkv, 128, 2000, r, ab.BF16, seed=Hq * 100 + r)
+    before = ab.ahakv_launch_count()
+    parity.run_evict(p, q, k, v)
+    assert ab.ahakv_launch_count() - before == 3
+    parity.check_units(p, q, k, v, parity.all_units(p))
+
+
 def test_peaked_attention_large_logits():
     """Queries 6x larger: logits reach the hundreds, single keys take almost all the mass."""
     B, Hq, Hkv, d, n, r = 1, 2, 2, 128, 900, 32
-    # float32 keeps its 1e-5 tolerance only while FP32 accumulation of the dot product does: logits
-    # of a few tens, not hundreds
-    for dtype, spread in ((ab.F16, 6.0), (ab.BF16, 6.0), (ab.F32, 2.0)):
+    # float32 inputs hold 1e-5 here too: their logits are formed, scaled and shifted in double
+    for dtype, spread in ((ab.F16, 6.0), (ab.BF16, 6.0), (ab.F32, 6.0)):
         p = ab.Params(B, Hq, Hkv, d, n, r, 16, 100, dtype=dtype, n_total=50000)
         q, k, v = _rand_problem(B, Hq, Hkv, d, n, r, dtype, seed=5, spread=spread)
         parity.check_units(p, q, k, v, parity.all_units(p))
