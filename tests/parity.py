@@ -91,14 +91,32 @@ def run_score(p: ab.Params, q, k, v, score_prev=None):
     return score
 
 
-def check_units(p: ab.Params, q, k, v, units, score_prev=None, nthreads=0):
+def oracle_units(p: ab.Params, q, k, v, units, score_prev=None, workers: int = 1):
+    """The oracle's eviction of each listed (b, h) unit, `workers` units at a time (one host thread each; the
+    oracle call releases the interpreter lock).  Yields (b, h, inputs, result) in the order given."""
+    units = list(units)
+
+    def one(bh):
+        inp = unit_inputs(p, q, k, v, bh[0], bh[1], score_prev)
+        return inp, orc.evict(*inp, nthreads=1)
+
+    if workers <= 1:
+        for bh in units:
+            inp, ref = one(bh)
+            yield bh[0], bh[1], inp, ref
+        return
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=workers) as ex:
+        for bh, (inp, ref) in zip(units, ex.map(one, units)):
+            yield bh[0], bh[1], inp, ref
+
+
+def check_units(p: ab.Params, q, k, v, units, score_prev=None, workers: int = 1):
     """Fused evict + separate score on the GPU, compared with the oracle on the listed (b, h) units."""
     score = run_score(p, q, k, v, score_prev)
     k_out, v_out, s_out, idx = run_evict(p, q, k, v, score_prev)
     stats = dict(max_rel=0.0, idx_diffs=0, units=0)
-    for b, h in units:
-        op, qn, kn, vn, sp = unit_inputs(p, q, k, v, b, h, score_prev)
-        ref = orc.evict(op, qn, kn, vn, sp, nthreads=nthreads)
+    for b, h, (op, qn, kn, vn, sp), ref in oracle_units(p, q, k, v, units, score_prev, workers):
         stats["max_rel"] = max(stats["max_rel"],
                                assert_scores_close(p, score[b, h].cpu().numpy(), ref["score"][0, 0]))
         gi = idx[b, h].cpu().numpy()
@@ -111,7 +129,28 @@ def check_units(p: ab.Params, q, k, v, units, score_prev=None, nthreads=0):
         assert torch.equal(s_out[b, h], score[b, h][idx[b, h].long()])
         assert_scores_close(p, s_out[b, h].cpu().numpy(), so[0, 0], "score_out")
         stats["units"] += 1
+    stats["outputs"] = (score, k_out, v_out, s_out, idx)
     return stats
+
+
+def assert_every_head_valid(p: ab.Params, idx, score_no_prior=None):
+    """Properties that hold at any size, checked on the device for every (sequence, KV head) of a launch:
+    kept indices strictly ascending, in range, exactly n_keep of them, recent window at the tail; and, for a
+    score computed without the value prior and without a carried score, sum_j S_j = r (each of the r softmax
+    rows carries mass 1; the mean over a group's query heads keeps it)."""
+    n, Br, n_keep = p.n_ctx, p.recent_window, p.n_keep
+    assert idx.shape == (p.batch, p.n_kv_heads, n_keep)
+    i64 = idx.long()
+    assert bool((i64[..., 1:] > i64[..., :-1]).all()), "kept indices must be strictly ascending in every head"
+    assert int(i64.min()) >= 0 and int(i64.max()) < n
+    if n > p.budget and Br > 0:
+        want = torch.arange(n - Br, n, device=idx.device).expand(p.batch, p.n_kv_heads, Br)
+        assert torch.equal(i64[..., n_keep - Br:], want), "recent window must close every head's kept list"
+    if score_no_prior is not None:
+        total = score_no_prior.double().sum(-1)
+        assert bool((score_no_prior >= 0).all())
+        assert torch.allclose(total, torch.full_like(total, float(p.obs_window)), rtol=2e-4), \
+            f"softmax mass: min {float(total.min())} max {float(total.max())} want {p.obs_window}"
 
 
 def all_units(p: ab.Params):
