@@ -54,7 +54,7 @@ typedef enum {
 enum {
   AHAKV_FLAG_VALUE_PRIOR = 1,   /* refine the score with Eq. 13-15                                   */
   AHAKV_FLAG_POOL_ZERO_PAD = 2, /* Eq. 13's mean filter divides edge windows by the full width        */
-  AHAKV_FLAG_GROUP_MAX = 4      /* pool grouped query heads by max instead of mean (not built yet)    */
+  AHAKV_FLAG_GROUP_MAX = 4      /* pool the query heads of a KV head by maximum instead of mean        */
 };
 
 typedef struct CUstream_st* ahakv_stream_t; /* a cudaStream_t; NULL is the legacy default stream */

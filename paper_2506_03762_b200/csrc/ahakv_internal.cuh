@@ -26,6 +26,7 @@ struct Shape {
   long long n_total;
   int R;          // G * r
   int n_blk;      // ceil(n / kKeyTile)
+  int group_max;  // pool the query heads of a KV head by maximum instead of mean (and G > 1)
   long long qs[3], ks[3], vs[3];  // element strides: batch, head, token
 };
 
@@ -52,12 +53,13 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
                              float2* partial, int* counters, int* status, cudaStream_t st);
 bool score_tc_available();
 ahakv_status launch_vnorm(const Plan& pl, const void* v, float* nu, cudaStream_t st);
+// `slots` partial scores per head (row blocks, or query heads when pooling by maximum) are combined here.
 ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
-                           float* score, cudaStream_t st);
+                           float* score, int slots, cudaStream_t st);
 ahakv_status launch_select(const Plan& pl, const float* score, int32_t* kept_idx, cudaStream_t st);
 bool refine_select_fits(const Plan& pl);
 ahakv_status launch_refine_select(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
-                                  float* score, int32_t* kept_idx, cudaStream_t st);
+                                  float* score, int32_t* kept_idx, int slots, cudaStream_t st);
 ahakv_status launch_compact(const Plan& pl, const void* k, const void* v, const float* score,
                             const int32_t* kept_idx, void* k_out, void* v_out, float* score_out,
                             cudaStream_t st);

@@ -56,7 +56,6 @@ ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
   if (p->flags & ~(uint32_t)(AHAKV_FLAG_VALUE_PRIOR | AHAKV_FLAG_POOL_ZERO_PAD | AHAKV_FLAG_GROUP_MAX))
     return AHAKV_ERR_INVALID_ARG;
   if ((long long)p->batch * p->n_kv_heads > 65535LL) return AHAKV_ERR_INVALID_ARG;
-  if (p->flags & AHAKV_FLAG_GROUP_MAX) return AHAKV_ERR_UNSUPPORTED;
 
   Plan& o = *pl;
   o.B = p->batch; o.Hq = p->n_q_heads; o.Hkv = p->n_kv_heads; o.G = G; o.d = p->head_dim;
@@ -66,6 +65,7 @@ ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
   o.dtype = p->dtype; o.es = p->dtype == AHAKV_F32 ? 4 : 2;
   o.pool = p->pool_kernel; o.flags = p->flags; o.n_total = p->n_total;
   o.R = G * p->obs_window;
+  o.group_max = (p->flags & AHAKV_FLAG_GROUP_MAX) != 0 && G > 1;   // the maximum over one head is that head
   o.n_blk = (o.n + kKeyTile - 1) / kKeyTile;
   if (!resolve_strides(p->q_stride, o.qs, o.Hq, o.r, o.d, o.es) ||
       !resolve_strides(p->k_stride, o.ks, o.Hkv, o.n, o.d, o.es) ||
@@ -90,6 +90,7 @@ ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
     if (o.r <= 128) {
       int hb = 128 / o.r;
       if (hb > G) hb = G;
+      if (o.group_max) hb = 1;     // one query head a row block: the blocks' scores are the per-head scores
       o.heads_per_rb = hb;
       o.n_rb = (G + hb - 1) / hb;
       o.use_tc = true;
@@ -123,11 +124,10 @@ static ahakv_status check_ws(const Plan& pl, void* ws, size_t ws_bytes) {
 
 template <typename T> static T* at(void* ws, size_t off) { return reinterpret_cast<T*>((char*)ws + off); }
 
-// Queues the scoring kernels; the refined score lands in `score`.  With `kept_idx` the selection is queued
-// too, in the same launch as the refinement when a head's scores fit in one CTA's registers.
-static ahakv_status queue_score(const Plan& pl, const void* q, const void* k, const void* v,
-                                const float* score_prev, float* score, int32_t* kept_idx, void* ws, cudaStream_t st,
-                                int prof) {
+// Queues the kernels that leave the raw accumulated score (per row block) and, with the value prior, the value
+// norms in the workspace.
+static ahakv_status queue_raw_score(const Plan& pl, const void* q, const void* k, const void* v, void* ws,
+                                    cudaStream_t st, int prof) {
   ahakv_status rc = cuda_ok(cudaMemsetAsync(at<char>(ws, pl.off_status), 0, pl.off_sraw - pl.off_status, st));
   if (rc) return rc;
   profile_mark(prof, 0, st);
@@ -148,16 +148,10 @@ static ahakv_status queue_score(const Plan& pl, const void* q, const void* k, co
     if (rc) return rc;
   }
   profile_mark(prof, 2, st);
-  if (kept_idx && refine_select_fits(pl)) {
-    rc = launch_refine_select(pl, s_raw, nu, score_prev, score, kept_idx, st);
-    profile_mark(prof, 3, st);
-    return rc;
-  }
-  rc = launch_refine(pl, s_raw, nu, score_prev, score, st);
-  profile_mark(prof, 3, st);
-  if (rc == AHAKV_OK && kept_idx) rc = launch_select(pl, score, kept_idx, st);
-  return rc;
+  return AHAKV_OK;
 }
+
+static int score_slots(const Plan& pl) { return pl.use_tc ? pl.n_rb : 1; }
 
 }  // namespace ahakv
 
@@ -189,9 +183,13 @@ ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k
     return AHAKV_ERR_INVALID_ARG;
   if ((rc = check_ws(pl, ws, ws_bytes))) return rc;
   const int prof = profile_begin_call((cudaStream_t)stream);
-  rc = queue_score(pl, q_obs, k, v, score_prev, score, nullptr, ws, (cudaStream_t)stream, prof);
-  profile_mark(prof, 4, (cudaStream_t)stream);   // no selection or compaction in this call
-  profile_mark(prof, 5, (cudaStream_t)stream);
+  cudaStream_t st = (cudaStream_t)stream;
+  if ((rc = queue_raw_score(pl, q_obs, k, v, ws, st, prof))) return rc;
+  rc = launch_refine(pl, at<float>(ws, pl.off_sraw), prior ? at<float>(ws, pl.off_nu) : nullptr, score_prev, score,
+                     score_slots(pl), st);
+  profile_mark(prof, 3, st);
+  profile_mark(prof, 4, st);   // no selection or compaction in this call
+  profile_mark(prof, 5, st);
   return rc;
 }
 
@@ -230,11 +228,22 @@ ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k
     return AHAKV_ERR_INVALID_ARG;
   if ((rc = check_ws(pl, ws, ws_bytes))) return rc;
   cudaStream_t st = (cudaStream_t)stream;
-  float* score = at<float>(ws, pl.off_score);
   const int prof = profile_begin_call(st);
-  if ((rc = queue_score(pl, q_obs, k, v, score_prev, score, kept_idx, ws, st, prof))) return rc;
+  if ((rc = queue_raw_score(pl, q_obs, k, v, ws, st, prof))) return rc;
+  const bool prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0;
+  float* s_raw = at<float>(ws, pl.off_sraw);
+  float* nu = prior ? at<float>(ws, pl.off_nu) : nullptr;
+  float* score = at<float>(ws, pl.off_score);
+  if (refine_select_fits(pl)) {      // a head's scores fit in one CTA's registers: both steps in one launch
+    rc = launch_refine_select(pl, s_raw, nu, score_prev, score, kept_idx, score_slots(pl), st);
+    profile_mark(prof, 3, st);
+  } else {
+    rc = launch_refine(pl, s_raw, nu, score_prev, score, score_slots(pl), st);
+    profile_mark(prof, 3, st);
+    if (rc == AHAKV_OK) rc = launch_select(pl, score, kept_idx, st);
+  }
   profile_mark(prof, 4, st);
-  rc = launch_compact(pl, k, v, score_out ? score : nullptr, kept_idx, k_out, v_out, score_out, st);
+  if (rc == AHAKV_OK) rc = launch_compact(pl, k, v, score_out ? score : nullptr, kept_idx, k_out, v_out, score_out, st);
   profile_mark(prof, 5, st);
   return rc;
 }

@@ -129,7 +129,7 @@ __global__ void simt_merge_stats(const float2* __restrict__ partial, float2* __r
       const float2 e = p[(size_t)t * pl.R];
       if (e.y > 0.f) Z += e.y * fast_exp2(e.x - M);
     }
-    final_st[(size_t)unit * pl.R + s] = make_float2(M, 1.f / (Z * (float)pl.G));
+    final_st[(size_t)unit * pl.R + s] = make_float2(M, 1.f / (Z * (float)(pl.group_max ? 1 : pl.G)));
   }
 }
 
@@ -151,13 +151,17 @@ __global__ void __launch_bounds__(kThreads) simt_column_sums(const T* __restrict
   if (j >= pl.n) return;
   float kreg[D];
   load_key<T, D>(k, pl, b, h, j, kreg);
-  float acc = 0.f;
+  float acc = 0.f, best = 0.f;
   for (int s = 0; s < pl.R; ++s) {
     const int i = s % pl.r;
+    if (pl.group_max && i == 0 && s > 0) {        // a query head is complete: keep the largest head's score
+      best = fmaxf(best, acc);
+      acc = 0.f;
+    }
     if (j <= pl.n - pl.r + i)
       acc = fmaf(fast_exp2((float)fma(dot_row<D, A>(qsm + s * D, kreg), cs.c[i], -(A)st[s].x)), st[s].y, acc);
   }
-  s_raw[(size_t)unit * pl.n + j] = acc;
+  s_raw[(size_t)unit * pl.n + j] = pl.group_max ? fmaxf(best, acc) : acc;
 }
 
 template <typename T, int D>

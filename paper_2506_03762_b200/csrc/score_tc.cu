@@ -154,6 +154,17 @@ __device__ __forceinline__ bool mbar_try(void* bar, int parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
+// The same without ever suspending the thread: for a thread that polls several barriers in turn and must not
+// sit on one while another has come free.
+__device__ __forceinline__ bool mbar_test(void* bar, int parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait.  Returns false (and records the timeout) if the phase did not complete in time.  The
 // clock is slow to read, so it is looked at only after many failed tries (each of which already sleeps in
 // hardware for a while).
@@ -486,7 +497,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
     }
     if (k_state == 1) {
       const int qb = sc & 1;
-      if (mbar_try(&bars->q_empty[qb], ((sc >> 1) & 1) ^ 1)) {
+      if (mbar_test(&bars->q_empty[qb], ((sc >> 1) & 1) ^ 1)) {
         char* q_smem = tiles + kOffQ + qb * kQBytes;
         mbar_expect_tx(&bars->q_full[qb], q_bytes);
         for (int s = 0; s < n_sub; ++s) {
@@ -499,7 +510,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
       }
     } else if (k_state == 2) {
       const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
-      if (mbar_try(&bars->k_empty[stage], ph ^ 1)) {
+      if (mbar_test(&bars->k_empty[stage], ph ^ 1)) {
         mbar_expect_tx(&bars->k_full[stage], k_bytes);
         char* dst = tiles + kOffK + stage * kKStageBytes;
         for (int s = 0; s < n_sub; ++s) {
@@ -519,7 +530,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
     }
     if (v_state == 2) {
       const int vs = vc % kVStages;
-      if (mbar_try(&bars->v_empty[vs], ((vc / kVStages) & 1) ^ 1)) {
+      if (mbar_test(&bars->v_empty[vs], ((vc / kVStages) & 1) ^ 1)) {
         mbar_expect_tx(&bars->v_full[vs], n_sub * kVSubBytes);
         char* dst = tiles + kOffV + vs * kVStageBytes;
         for (int s = 0; s < n_sub; ++s)
@@ -1136,7 +1147,7 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   const int grid = a.n_runs < n_sm ? a.n_runs : n_sm;
   a.bf16 = pl.dtype == AHAKV_BF16;
   a.prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0 && v != nullptr && nu != nullptr;
-  a.log2G = log2f((float)pl.G);
+  a.log2G = pl.group_max ? 0.f : log2f((float)pl.G);   // pooling by maximum keeps each head's own score
   for (int i = 0; i < kMaxRows; ++i) a.c[i] = pl.rows.c[i];
   for (int t = 0; t < 128; ++t) a.cs[t] = pl.r <= 128 ? pl.rows.c[t % pl.r] : 0.f;
   a.partial = reinterpret_cast<float*>(partial_ws); a.s_raw = s_raw; a.nu = nu;

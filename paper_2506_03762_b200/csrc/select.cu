@@ -8,6 +8,7 @@
 //   the float, then emits, in ascending index order, every candidate above the
 //   threshold plus the lowest-indexed ones equal to it, then the recent window.
 #include "ahakv_internal.cuh"
+#include "select_common.cuh"
 
 namespace ahakv {
 namespace {
@@ -26,48 +27,27 @@ __device__ __forceinline__ float block_max(float x, float* red) {
   return m;
 }
 
-__device__ __forceinline__ float pooled(const float* __restrict__ nu, int j, int n, int half, float inv_full) {
-  const int lo = max(j - half, 0), hi = min(j + half, n - 1);
-  float s;
-  if (hi - lo == 6) {
-    // the usual width (7) away from the ends: seven independent loads, added in the order of the loop below
-    const float a0 = nu[lo], a1 = nu[lo + 1], a2 = nu[lo + 2], a3 = nu[lo + 3], a4 = nu[lo + 4], a5 = nu[lo + 5],
-                a6 = nu[lo + 6];
-    s = (((((a0 + a1) + a2) + a3) + a4) + a5) + a6;
-  } else {
-    s = 0.f;
-    for (int t = lo; t <= hi; ++t) s += nu[t];
-  }
-  return inv_full > 0.f ? s * inv_full : s / (float)(hi - lo + 1);
-}
-
 __global__ void __launch_bounds__(kThreads) refine_kernel(const float* __restrict__ s_raw, const float* __restrict__ nu,
                                                           const float* __restrict__ prev, float* __restrict__ score,
                                                           const Shape pl, const int slots) {
   __shared__ float red[kWarps];
   const int unit = blockIdx.x, n = pl.n, half = pl.pool / 2;
   const bool prior = nu != nullptr;
-  const float inv_full = (pl.flags & AHAKV_FLAG_POOL_ZERO_PAD) ? 1.f / (float)pl.pool : 0.f;
+  const float inv_w = 1.f / (float)pl.pool;
+  const bool zero_pad = (pl.flags & AHAKV_FLAG_POOL_ZERO_PAD) != 0;
   const float* nu_u = prior ? nu + (size_t)unit * n : nullptr;
-  float gmax = 1.f;
+  float inv_gmax = 1.f;
   if (prior) {
     float m = 0.f;
-    for (int j = threadIdx.x; j < n; j += kThreads) m = fmaxf(m, pooled(nu_u, j, n, half, inv_full));
-    gmax = block_max(m, red);
+    for (int j = threadIdx.x; j < n; j += kThreads) m = fmaxf(m, pooled(nu_u, j, n, half, inv_w, zero_pad));
+    inv_gmax = __frcp_rn(block_max(m, red));
   }
   for (int j = threadIdx.x; j < n; j += kThreads) {
-    float s = s_raw[(size_t)unit * slots * n + j];
-    for (int t = 1; t < slots; ++t) s += s_raw[((size_t)unit * slots + t) * n + j];
-    if (prior) s = __fmul_rn(__fdiv_rn(pooled(nu_u, j, n, half, inv_full), gmax), s);
+    float s = combine_slots(s_raw, (size_t)unit * slots * n + j, n, slots, pl.group_max);
+    if (prior) s = __fmul_rn(__fmul_rn(pooled(nu_u, j, n, half, inv_w, zero_pad), inv_gmax), s);
     if (prev) s = __fadd_rn(s, prev[(size_t)unit * n + j]);
     score[(size_t)unit * n + j] = s;
   }
-}
-
-// Monotone map float -> uint32: a > b  <=>  key(a) > key(b) (for non-NaN values).
-__device__ __forceinline__ uint32_t order_key(float x) {
-  const uint32_t u = __float_as_uint(x);
-  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
 // The digit at which the count of keys, taken from the largest digit down, reaches `need`: a suffix scan of
@@ -189,11 +169,12 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
   const int unit = blockIdx.x, n = pl.n, half = pl.pool / 2;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const bool prior = nu != nullptr;
-  const float inv_full = (pl.flags & AHAKV_FLAG_POOL_ZERO_PAD) ? 1.f / (float)pl.pool : 0.f;
+  const float inv_w = 1.f / (float)pl.pool;
+  const bool zero_pad = (pl.flags & AHAKV_FLAG_POOL_ZERO_PAD) != 0;
   const float* nu_u = prior ? nu + (size_t)unit * n : nullptr;
 
   uint32_t key[kPer];                                       // first the bits of gamma, then the score's order key
-  float gmax = 1.f;
+  float inv_gmax = 1.f;
   if (prior) {
     // the head's value norms go to shared memory in one coalesced sweep; the mean filter reads them there
     extern __shared__ float nu_s[];
@@ -215,11 +196,11 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
 #pragma unroll
     for (int e = 0; e < kPer; ++e) {
       const int j = e * kThreads + threadIdx.x;
-      const float g = j < n ? pooled(nu_s, j, n, half, inv_full) : 0.f;
+      const float g = j < n ? pooled(nu_s, j, n, half, inv_w, zero_pad) : 0.f;
       key[e] = __float_as_uint(g);
       m = fmaxf(m, g);
     }
-    gmax = block_max(m, red);
+    inv_gmax = __frcp_rn(block_max(m, red));
   }
   // loads in flight at a time: without a carried score, and with fewer than 32 keys to hold, the registers allow
   // twice as many
@@ -233,8 +214,7 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
       const int j = (e0 + e) * kThreads + threadIdx.x;
       sr[e] = 0.f; pv[e] = 0.f;
       if (j < n) {
-        sr[e] = s_raw[(size_t)unit * slots * n + j];
-        for (int t = 1; t < slots; ++t) sr[e] += s_raw[((size_t)unit * slots + t) * n + j];
+        sr[e] = combine_slots(s_raw, (size_t)unit * slots * n + j, n, slots, pl.group_max);
         if (kPrev) pv[e] = prev[(size_t)unit * n + j];
       }
     }
@@ -245,7 +225,7 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
       key[e0 + e] = 0u;
       if (j < n) {
         float s = sr[e];
-        if (prior) s = __fmul_rn(__fdiv_rn(g, gmax), s);
+        if (prior) s = __fmul_rn(__fmul_rn(g, inv_gmax), s);
         if (kPrev) s = __fadd_rn(s, pv[e]);
         score[(size_t)unit * n + j] = s;
         key[e0 + e] = order_key(s);
@@ -276,11 +256,19 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
     for (int e = 0; e < kPer; ++e) {
       const bool in = e * kThreads + (int)threadIdx.x < n_cand && (key[e] & mask) == prefix;
       const unsigned digit = (key[e] >> shift) & 255u;
-      // one atomic per distinct digit of the warp
-      const unsigned live = __ballot_sync(0xffffffffu, in);
-      if (in) {
-        const unsigned same = __match_any_sync(live, digit);
-        if (lane == __ffs(same) - 1) atomicAdd(&hist[warp & (kHistCopies - 1)][digit], (unsigned)__popc(same));
+      unsigned* bins = hist[warp & (kHistCopies - 1)];
+      if (pass == 0) {
+        // sign and high exponent bits: nearly all scores of a head share one digit, and atomics on one counter
+        // are served one after the other.  One atomic for the warp when all its digits agree.
+        const unsigned live = __ballot_sync(0xffffffffu, in);
+        const unsigned first = __shfl_sync(0xffffffffu, digit, live ? __ffs(live) - 1 : 0);
+        if (__all_sync(0xffffffffu, !in || digit == first)) {
+          if (live && lane == __ffs(live) - 1) atomicAdd(&bins[digit], (unsigned)__popc(live));
+        } else if (in) {
+          atomicAdd(&bins[digit], 1u);
+        }
+      } else if (in) {                         // later digits are spread out, and ever fewer tokens are still in
+        atomicAdd(&bins[digit], 1u);
       }
     }
     __syncthreads();
@@ -334,8 +322,8 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
 }  // namespace
 
 ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
-                           float* score, cudaStream_t st) {
-  refine_kernel<<<pl.B * pl.Hkv, kThreads, 0, st>>>(s_raw, nu, score_prev, score, pl, pl.use_tc ? pl.n_rb : 1);
+                           float* score, int slots, cudaStream_t st) {
+  refine_kernel<<<pl.B * pl.Hkv, kThreads, 0, st>>>(s_raw, nu, score_prev, score, pl, slots);
   count_launch();
   return cuda_ok(cudaGetLastError());
 }
@@ -353,7 +341,7 @@ bool refine_select_fits(const Plan& pl) { return pl.n <= kPerMax * kThreads; }
 namespace {
 template <int kPer, bool kPrev>
 ahakv_status launch_refine_select_as(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
-                                     float* score, int32_t* kept_idx, cudaStream_t st) {
+                                     float* score, int32_t* kept_idx, int slots, cudaStream_t st) {
   // Static and dynamic shared memory together may pass 48 KB well before the dynamic part alone does, and
   // beyond that the launch needs leave, asked for once per device: ask whenever the value norms are staged.
   constexpr int kMaxDevices = 64;
@@ -370,25 +358,25 @@ ahakv_status launch_refine_select_as(const Plan& pl, const float* s_raw, const f
     }
   }
   refine_select_kernel<kPer, kPrev><<<pl.B * pl.Hkv, kThreads, smem, st>>>(s_raw, nu, score_prev, score, kept_idx, pl,
-                                                                    pl.use_tc ? pl.n_rb : 1);
+                                                                    slots);
   count_launch();
   return cuda_ok(cudaGetLastError());
 }
 }  // namespace
 
 ahakv_status launch_refine_select(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
-                                  float* score, int32_t* kept_idx, cudaStream_t st) {
+                                  float* score, int32_t* kept_idx, int slots, cudaStream_t st) {
   const int per = (pl.n + kThreads - 1) / kThreads;          // tokens a thread owns
   if (score_prev) {
-    if (per <= 4) return launch_refine_select_as<4, true>(pl, s_raw, nu, score_prev, score, kept_idx, st);
-    if (per <= 8) return launch_refine_select_as<8, true>(pl, s_raw, nu, score_prev, score, kept_idx, st);
-    if (per <= 16) return launch_refine_select_as<16, true>(pl, s_raw, nu, score_prev, score, kept_idx, st);
-    return launch_refine_select_as<kPerMax, true>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+    if (per <= 4) return launch_refine_select_as<4, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
+    if (per <= 8) return launch_refine_select_as<8, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
+    if (per <= 16) return launch_refine_select_as<16, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
+    return launch_refine_select_as<kPerMax, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
   }
-  if (per <= 4) return launch_refine_select_as<4, false>(pl, s_raw, nu, score_prev, score, kept_idx, st);
-  if (per <= 8) return launch_refine_select_as<8, false>(pl, s_raw, nu, score_prev, score, kept_idx, st);
-  if (per <= 16) return launch_refine_select_as<16, false>(pl, s_raw, nu, score_prev, score, kept_idx, st);
-  return launch_refine_select_as<kPerMax, false>(pl, s_raw, nu, score_prev, score, kept_idx, st);
+  if (per <= 4) return launch_refine_select_as<4, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
+  if (per <= 8) return launch_refine_select_as<8, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
+  if (per <= 16) return launch_refine_select_as<16, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
+  return launch_refine_select_as<kPerMax, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
 }
 
 }  // namespace ahakv

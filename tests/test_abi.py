@@ -87,8 +87,7 @@ def test_bad_pointers_and_workspace_are_rejected_on_the_host(lib):
     assert ab.ahakv_compact(p, 256, None, None, 256, 256, 256, None, stream=0, check=False) == ab.ERR_INVALID_ARG
     assert ab.ahakv_evict(p, 256, 256, 256, None, 256, 256, None, None, 256, need, stream=0,
                           check=False) == ab.ERR_INVALID_ARG
-    assert ab.ahakv_score(_good(flags=ab.FLAG_GROUP_MAX), 256, 256, 256, None, 256, 256, need, stream=0,
-                          check=False) == ab.ERR_UNSUPPORTED
+    assert ab.ahakv_workspace_bytes(_good(flags=ab.FLAG_GROUP_MAX)) > 0      # pooling by maximum is a legal request
 
 
 def test_status_strings_and_errors(lib):

@@ -163,6 +163,11 @@ EDGE_CASES = [
     (1, 2, 1, 64, 11000, 16, 32, 900, ab.BF16, {}),
     (1, 1, 1, 64, 12288, 16, 32, 900, ab.F16, {}),
     (1, 1, 1, 64, 12288, 16, 32, 900, ab.BF16, dict(n_total=40000)),
+    # grouped query heads pooled by maximum instead of mean
+    (1, 8, 2, 128, 1500, 32, 16, 300, ab.F16, dict(flags=ab.FLAG_VALUE_PRIOR | ab.FLAG_GROUP_MAX)),
+    (2, 8, 2, 128, 700, 64, 16, 200, ab.BF16, dict(flags=ab.FLAG_GROUP_MAX)),
+    (1, 6, 2, 64, 400, 20, 8, 100, ab.F32, dict(flags=ab.FLAG_VALUE_PRIOR | ab.FLAG_GROUP_MAX)),
+    (1, 2, 2, 128, 600, 200, 16, 150, ab.F16, dict(flags=ab.FLAG_GROUP_MAX)),     # one head a group: same as the mean
     # query heads that do not fill the last row block of their KV head
     (1, 7, 1, 128, 1300, 32, 32, 300, ab.BF16, {}),                        # G = 7, r = 32: blocks of 4 + 3 heads
     (2, 14, 2, 128, 1300, 32, 32, 300, ab.F16, {}),
