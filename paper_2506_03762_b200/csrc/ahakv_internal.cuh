@@ -52,6 +52,12 @@ ahakv_status launch_score_simt(const Plan& pl, const void* q, const void* k, flo
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
                              float2* partial, int* counters, int* status, cudaStream_t st);
 bool score_tc_available();
+// The tensor-core kernel that keeps the softmax numerators in tensor memory (score_res.cu): each key tile is
+// fetched, multiplied and exponentiated once.  `partial` holds one float per (row block, tile, row), `lfin` one
+// per (row block, row).  Takes the problems score_res_fits() accepts; the two-pass kernel takes the others.
+bool score_res_fits(const Plan& pl);
+ahakv_status launch_score_res(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
+                              float* partial, float* lfin, int* status, cudaStream_t st);
 ahakv_status launch_vnorm(const Plan& pl, const void* v, float* nu, cudaStream_t st);
 // `slots` partial scores per head (row blocks, or query heads when pooling by maximum) are combined here.
 ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,

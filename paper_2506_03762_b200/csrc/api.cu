@@ -2,6 +2,7 @@
 // layout and the order in which the kernels are queued.
 #include <atomic>
 #include <cmath>
+#include <cstdlib>
 #include <cstring>
 
 #include "ahakv_internal.cuh"
@@ -136,7 +137,11 @@ static ahakv_status queue_raw_score(const Plan& pl, const void* q, const void* k
   float* final_off = at<float>(ws, pl.off_final);
   const bool prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0;
   float* nu = prior ? at<float>(ws, pl.off_nu) : nullptr;
-  if (pl.use_tc)   // the tensor-core kernel squares the value rows on its way
+  static const bool two_pass_only = std::getenv("AHAKV_TWO_PASS_SCORING") != nullptr;   // measurement switch
+  if (pl.use_tc && !two_pass_only && score_res_fits(pl))   // the tensor-core kernels square the value rows on their way
+    rc = launch_score_res(pl, q, k, prior ? v : nullptr, s_raw, nu, reinterpret_cast<float*>(partial), final_off,
+                          at<int>(ws, pl.off_status), st);
+  else if (pl.use_tc)
     rc = launch_score_tc(pl, q, k, prior ? v : nullptr, s_raw, nu, partial, at<int>(ws, pl.off_sync),
                          at<int>(ws, pl.off_status), st);
   else

@@ -58,9 +58,12 @@
 #include <cuda.h>
 
 #include "ahakv_internal.cuh"
+#include "tc_common.cuh"
 
 namespace ahakv {
 namespace {
+
+using namespace tc;
 
 constexpr int kKStages = 3;                // K-tile ring depth
 constexpr int kSubTileBytes = 128 * 128;   // 128 rows x 64 16-bit elements, 128-byte swizzled
@@ -72,7 +75,6 @@ constexpr int kSegAhead = 4;               // segments published beyond the one 
 constexpr int kSegEnd = -1;
 constexpr int kVSubBytes = kVRows * 128;
 constexpr int kThreads = 768;              // TMA + scheduler warp, MMA warp, 2 merge warps, 16 softmax warps, 4 value-norm warps
-constexpr long long kWaitLimitNs = 1000000000LL;   // 1 s
 constexpr float kFold = 256.f;             // value of the constant tile; offsets are stored divided by it
 
 struct TcArgs {
@@ -127,159 +129,6 @@ constexpr int kSmemTiles = kOffExt + 3 * kExtBytes;      // 204 KiB
 constexpr int kSmemBytes = kSmemTiles + 1024 /*alignment slack*/ + 13312 /*barriers, constants, exchange*/;
 static_assert(sizeof(Shared) <= 13312, "Shared outgrew its reservation");
 
-// ---- PTX wrappers ------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ long long now_ns() {
-  long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-
-__device__ __forceinline__ void mbar_init(void* bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(void* bar, int bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(void* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(void* bar, int parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// The same without ever suspending the thread: for a thread that polls several barriers in turn and must not
-// sit on one while another has come free.
-__device__ __forceinline__ bool mbar_test(void* bar, int parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false (and records the timeout) if the phase did not complete in time.  The
-// clock is slow to read, so it is looked at only after many failed tries (each of which already sleeps in
-// hardware for a while).
-__device__ __forceinline__ bool mbar_wait(void* bar, int parity, int* status) {
-#pragma unroll 1
-  for (int t = 0; t < 256; ++t)
-    if (mbar_try(bar, parity)) return true;
-  const long long t0 = now_ns();
-  for (;;) {
-#pragma unroll 1
-    for (int t = 0; t < 256; ++t)
-      if (mbar_try(bar, parity)) return true;
-    if (now_ns() - t0 > kWaitLimitNs) {
-      atomicExch(status, (int)AHAKV_ERR_TIMEOUT);
-      return false;
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2,
-                                            int c3) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-      : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(void* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-
-// Shared-memory operand descriptor (fields as described at umma_desc_lo below) of a K-major tile of 32-byte
-// rows (16 elements, one k-step), 32-byte swizzle, 8-row groups 256 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc_ext(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr & 0x3ffff) >> 4);
-  d |= (uint64_t)1 << 16;
-  d |= (uint64_t)(256 >> 4) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)6 << 61;                               // SWIZZLE_32B
-  return d;
-}
-
-// Instruction descriptor for kind::f16: FP32 accumulate, A and B both K-major and of one type.
-__device__ __forceinline__ uint32_t umma_idesc(int M, int N, int bf16) {
-  uint32_t d = 0;
-  d |= 1u << 4;                         // D format F32
-  d |= (uint32_t)(bf16 ? 1 : 0) << 7;   // A format
-  d |= (uint32_t)(bf16 ? 1 : 0) << 10;  // B format
-  d |= (uint32_t)(N >> 3) << 17;
-  d |= (uint32_t)(M >> 4) << 24;
-  return d;
-}
-
-// 32 consecutive FP32 columns of this thread's TMEM lane: issue now, use after tmem_ld_wait(r).
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-// Waits for every TMEM load this thread has issued.  The registers pass through the statement, so no
-// use of them can be scheduled above the wait.
-__device__ __forceinline__ void tmem_ld_wait(uint32_t* r) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-                 "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-                 "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-               :
-               : "memory");
-}
-
-// 16 consecutive FP32 columns of this thread's TMEM lane: issue now, use after tmem_ld_wait16(r).
-__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait16(uint32_t* r) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
-               :
-               : "memory");
-}
-
-__device__ __forceinline__ void group_sync(int id, int threads) {
-  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-
-// One partial, straight from L2 (other CTAs write it while this one polls).
-__device__ __forceinline__ float2 ld_partial2(const float2* p) {   // two adjacent rows
-  float2 v;
-  asm volatile("ld.relaxed.gpu.global.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
-  return v;
-}
-__device__ __forceinline__ void st_partial(float* p, float v) {
-  asm volatile("st.relaxed.gpu.global.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
-}
-
 // ---- work decomposition ----------------------------------------------------------------------------------
 // A run = up to CH consecutive key tiles of one row block.  Every role of a CTA walks the runs its scheduler
 // has taken, in the order of the CTA's segment ring.
@@ -315,20 +164,6 @@ __device__ __forceinline__ UnitInfo unit_info(const TcArgs& a, int unit) {
 // Observation row index (0 .. r-1) of stacked row s of a row block.
 __device__ __forceinline__ int obs_row(const TcArgs& a, const UnitInfo& u, int s) {
   return a.r <= 128 ? s % a.r : u.rb * 128 + s;
-}
-
-__device__ __forceinline__ void tma_load_4d_hint(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2,
-                                                 int c3, unsigned long long policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-      " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
-      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy)
-      : "memory");
-}
-__device__ __forceinline__ unsigned long long policy_evict_first() {
-  unsigned long long p;
-  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-  return p;
 }
 
 // ---- the CTA's sequence of segments -------------------------------------------------------------------
@@ -599,30 +434,6 @@ __device__ void v_group(const TcArgs& a, Shared* sh, char* tiles) {
   if (leader) *(volatile int*)&sh->seg_done_v = 0x3fffffff;
 }
 
-// Shared-memory operand descriptor of a K-major tile of 128-byte rows with 128-byte swizzle: start address
-// (bits 0-13, in 16-byte units), leading byte offset (bits 16-29, unused with swizzle, set to 1), stride byte
-// offset between 8-row groups (bits 32-45: 1024 bytes), descriptor version 1 of sm_100 (bit 46), swizzle mode
-// (bits 61-63: 2 = 128 bytes).  Only the address field differs between the k-steps of a tile, so the low word
-// is made per tile and a k-step costs one add per operand; the high word is a constant.
-__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr) { return ((smem_addr & 0x3ffff) >> 4) | (1u << 16); }
-constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
-  uint64_t d;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
-  return d;
-}
-
-template <int ACC>
-__device__ __forceinline__ void umma_step(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc) {
-  const uint32_t accumulate = ACC;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
 // MMA issuer (one thread).
 // Pass 1: D[rows x keys] = Q K^T.  Pass 2: D[keys x rows] = K Q^T - off / c.
 __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tmem_base) {
@@ -678,27 +489,6 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tm
     }
     ++sc;
   });
-}
-
-// Two FP32 operations an instruction (packed f32x2 on 64-bit register pairs): the softmax warps are bound by
-// the number of instructions they issue, and every pair of adds or multiply-adds done this way is one less.
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
 }
 
 // One 32-key chunk of a row: fold it into the running pair (M, Z) with Z = sum of 2^{c w - M}.
@@ -1086,35 +876,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
 }
 
 // ---- host ------------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      return nullptr;
-    return reinterpret_cast<EncodeTiledFn>(p);
-  }();
-  return fn;
-}
-
-// 4-D map {d, tokens, heads, batch} with a {64, box_rows, box_heads, 1} box, 128-byte swizzle, zero fill.
-bool make_map(CUtensorMap* m, const void* base, int bf16, int d, long long tokens, long long heads, long long batch,
-              const long long stride[3], int es, int box_rows, int box_heads) {
-  const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)tokens, (cuuint64_t)heads, (cuuint64_t)batch};
-  const cuuint64_t strides[3] = {(cuuint64_t)stride[2] * es, (cuuint64_t)stride[1] * es, (cuuint64_t)stride[0] * es};
-  const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_heads, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return encode_fn()(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4,
-                     const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 }  // namespace
 
 bool score_tc_available() { return encode_fn() != nullptr; }
