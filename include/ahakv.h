@@ -98,6 +98,28 @@ ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k
                          const float* score_prev, float* score, void* ws, size_t ws_bytes,
                          ahakv_stream_t stream);
 
+/* The same score with the r observation rows at positions of the caller's choice instead of the last r (the
+ * paper's Limitations section: the recent rows are one choice of "a constant number of accumulators", a TopK
+ * choice of the same number another; which rows to take is the caller's policy, this entry point accumulates
+ * whichever it is given).  obs_pos: HOST array of r logical positions, strictly ascending, each inside the cache
+ * ([n_total - n_ctx, n_total)); q_obs holds the queries of those positions in that order.  Row i sees the cache
+ * rows up to its own position (Eq. 1) and, with AHAKV_SCALE_ADAPTIVE_ROW, takes Eq. 12 at obs_pos[i] + 1 tokens.
+ * obs_pos = the last r positions gives ahakv_score exactly. */
+ahakv_status ahakv_score_rows(const ahakv_params* p, const int64_t* obs_pos, const void* q_obs, const void* k,
+                              const void* v, const float* score_prev, float* score, void* ws, size_t ws_bytes,
+                              ahakv_stream_t stream);
+
+/* Accumulation over ALL query rows (Section 4.1, Eq. 2-3: S_j = sum over i >= j of a_ij; the paper's "w/o RA"
+ * ablation, and H2O's score when scale_mode is AHAKV_SCALE_FIXED with scale 1/sqrt(d) and the value prior is off).
+ * q_all holds a query for every cached row, [B,Hq,n,d] (q_stride describes it otherwise).  The rows are scored
+ * obs_window at a time (1 .. 256 / G; ceil(n / obs_window) passes of the kernels of ahakv_score, each over the
+ * keys its rows can see), summed, and the value prior and score_prev are applied to the sum.  O(n^2 d) work: this
+ * is the cost Recent Accumulation removes.  ws as for ahakv_score with the same parameters.
+ * AHAKV_FLAG_GROUP_MAX is not offered here (AHAKV_ERR_UNSUPPORTED). */
+ahakv_status ahakv_score_full_causal(const ahakv_params* p, const void* q_all, const void* k, const void* v,
+                                     const float* score_prev, float* score, void* ws, size_t ws_bytes,
+                                     ahakv_stream_t stream);
+
 /* Selection (Algorithm 1: S^r = recent B_r tokens, S^s = TopK(F, B_s), S = S^s U S^r).
  * Keeps rows [n - B_r, n) and the B_s = budget - B_r highest-scoring rows of [0, n - B_r);
  * equal scores are taken lowest index first; the result is ascending.  n <= budget keeps all rows.

@@ -64,6 +64,10 @@ typedef struct {
   double scale;           // lambda when scale_mode == FIXED
   int32_t pool_kernel;    // odd width of the mean filter
   uint32_t flags;
+  // Optional: the logical positions of the r observation rows, strictly ascending, each inside the cache
+  // ([n_total - n_ctx, n_total)).  NULL = the last r positions (Eq. 5).  With positions given, row i sees the
+  // cache rows up to its own position (Eq. 1's causal mask) and Eq. 12 counts the tokens up to it.
+  const int64_t* obs_pos;
 } oracle_params;
 
 }  // extern "C"
@@ -94,12 +98,22 @@ double load_elem(const void* p, int dtype, size_t idx) {
 }
 size_t elem_size(int dtype) { return dtype == ORACLE_F32 ? 4 : 2; }
 
+bool positions_ok(const oracle_params* p) {
+  if (!p->obs_pos) return true;
+  for (int i = 0; i < p->obs_window; ++i) {
+    if (p->obs_pos[i] < p->n_total - p->n_ctx || p->obs_pos[i] >= p->n_total) return false;
+    if (i > 0 && p->obs_pos[i] <= p->obs_pos[i - 1]) return false;
+  }
+  return true;
+}
+
 bool params_ok(const oracle_params* p) {
   return p && p->batch > 0 && p->n_q_heads > 0 && p->n_kv_heads > 0 && p->head_dim > 0 &&
          p->n_q_heads % p->n_kv_heads == 0 && p->n_ctx > 0 && p->n_total >= p->n_ctx &&
          p->obs_window >= 1 && p->obs_window <= p->n_ctx && p->budget >= 1 &&
          p->recent_window >= 0 && p->recent_window <= p->budget && p->dtype >= 0 && p->dtype <= 2 &&
-         p->scale_mode >= 0 && p->scale_mode <= 2 && p->pool_kernel >= 1 && (p->pool_kernel & 1);
+         p->scale_mode >= 0 && p->scale_mode <= 2 && p->pool_kernel >= 1 && (p->pool_kernel & 1) &&
+         positions_ok(p);
 }
 
 // Eq. 12: lambda = sqrt(2 log(i/k) / d); outside its domain fall back to 1/sqrt(d).
@@ -109,13 +123,17 @@ double eq12_lambda(double i_tokens, double k_budget, int d) {
   return std::sqrt(2.0 * std::log(ratio) / (double)d);
 }
 
-// lambda for observation row i (0-based among the r rows); its logical position
-// is p_i = n_total - r + i, so it has seen p_i + 1 tokens.
+// Logical position of observation row i (0-based among the r rows): the last r positions unless given.
+int64_t row_position(const oracle_params* p, int i) {
+  return p->obs_pos ? p->obs_pos[i] : p->n_total - p->obs_window + i;
+}
+
+// lambda for observation row i; at logical position p_i it has seen p_i + 1 tokens.
 double row_lambda(const oracle_params* p, int i) {
   switch (p->scale_mode) {
     case ORACLE_SCALE_FIXED: return p->scale;
     case ORACLE_SCALE_ADAPTIVE_ROW:
-      return eq12_lambda((double)(p->n_total - p->obs_window + i + 1), (double)p->budget, p->head_dim);
+      return eq12_lambda((double)(row_position(p, i) + 1), (double)p->budget, p->head_dim);
     default: return eq12_lambda((double)p->n_total, (double)p->budget, p->head_dim);
   }
 }
@@ -132,8 +150,9 @@ std::vector<double> widen(const void* p, int dtype, size_t off, size_t count) {
 // widened.  a[j] = 0 for masked columns.
 void attention_row(const oracle_params* p, const double* qrow, const double* kmat, int i,
                    std::vector<double>& a) {
-  const int n = p->n_ctx, r = p->obs_window, d = p->head_dim;
-  const int last = n - r + i;  // row i sees cache columns 0 .. n - r + i
+  const int n = p->n_ctx, d = p->head_dim;
+  // row i sees the cache columns up to its own position: n - r + i for the last r positions
+  const int last = (int)(row_position(p, i) - (p->n_total - p->n_ctx));
   const double lam = row_lambda(p, i);
   a.assign(n, 0.0);
   std::vector<double> x(last + 1);

@@ -42,6 +42,7 @@ class _Params(ctypes.Structure):
         ("obs_window", ctypes.c_int32), ("recent_window", ctypes.c_int32), ("budget", ctypes.c_int32),
         ("dtype", ctypes.c_int32), ("scale_mode", ctypes.c_int32), ("scale", ctypes.c_double),
         ("pool_kernel", ctypes.c_int32), ("flags", ctypes.c_uint32),
+        ("obs_pos", ctypes.POINTER(ctypes.c_int64)),
     ]
 
 
@@ -61,12 +62,20 @@ class OracleParams:
     scale: float = 0.0
     pool_kernel: int = 7
     flags: int = FLAG_VALUE_PRIOR
+    obs_pos: object = None              # None: the last r positions; else r ascending logical positions
 
     def c(self) -> _Params:
         nt = self.n_ctx if self.n_total is None else self.n_total
+        pos = None
+        if self.obs_pos is not None:
+            arr = np.ascontiguousarray(self.obs_pos, np.int64)
+            if arr.shape != (self.obs_window,):
+                raise ValueError("obs_pos must hold obs_window positions")
+            self._pos_keepalive = arr               # the C struct only borrows the pointer
+            pos = arr.ctypes.data_as(ctypes.POINTER(ctypes.c_int64))
         return _Params(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.n_ctx, nt,
                        self.obs_window, self.recent_window, self.budget, self.dtype, self.scale_mode,
-                       float(self.scale), self.pool_kernel, self.flags)
+                       float(self.scale), self.pool_kernel, self.flags, pos)
 
     @property
     def n_keep(self) -> int:

@@ -83,6 +83,8 @@ SIGNATURES = {
     "ahakv_workspace_bytes": (_sz, [_PP]),
     "ahakv_lambda": (ctypes.c_double, [ctypes.c_int64, ctypes.c_int32, ctypes.c_int32]),
     "ahakv_score": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_score_rows": (ctypes.c_int, [_PP, ctypes.POINTER(ctypes.c_int64), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_score_full_causal": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_select": (ctypes.c_int, [_PP, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_compact": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_evict": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -159,6 +161,31 @@ def ahakv_score(p: Params, q_obs, k, v, score_prev, score, ws, ws_bytes: int | N
                            _ptr(ws), nbytes, _stream(stream))
     if check:
         _raise(st, "ahakv_score")
+    return st
+
+
+def ahakv_score_rows(p: Params, obs_pos, q_obs, k, v, score_prev, score, ws, ws_bytes: int | None = None,
+                     stream=None, check: bool = True) -> int:
+    """``ahakv_score`` with the observation rows at the given logical positions (a host sequence of r ints)."""
+    cp = p.c()
+    pos = None if obs_pos is None else (ctypes.c_int64 * len(obs_pos))(*[int(x) for x in obs_pos])
+    nbytes = ws.numel() * ws.element_size() if ws_bytes is None else ws_bytes
+    st = lib().ahakv_score_rows(ctypes.byref(cp), pos, _ptr(q_obs), _ptr(k), _ptr(v), _ptr(score_prev),
+                                _ptr(score), _ptr(ws), nbytes, _stream(stream))
+    if check:
+        _raise(st, "ahakv_score_rows")
+    return st
+
+
+def ahakv_score_full_causal(p: Params, q_all, k, v, score_prev, score, ws, ws_bytes: int | None = None,
+                            stream=None, check: bool = True) -> int:
+    """Accumulation over all query rows (Eq. 2-3); ``p.obs_window`` rows per pass."""
+    cp = p.c()
+    nbytes = ws.numel() * ws.element_size() if ws_bytes is None else ws_bytes
+    st = lib().ahakv_score_full_causal(ctypes.byref(cp), _ptr(q_all), _ptr(k), _ptr(v), _ptr(score_prev),
+                                       _ptr(score), _ptr(ws), nbytes, _stream(stream))
+    if check:
+        _raise(st, "ahakv_score_full_causal")
     return st
 
 

@@ -37,12 +37,16 @@ struct Plan : Shape {
   bool use_tc;    // tensor-core scoring path applies
   RowScale rows;
   double lambda[kMaxRows];   // lambda_i itself, in double (the float32 path scales its logits in double)
+  int last[kMaxRows];        // per observation row: the last cache row it may see (n - r + i unless positions are given)
+  int n_eff;                 // last[r - 1] + 1: keys beyond are seen by no row
   // workspace layout, byte offsets
   size_t off_status, off_sync, off_sraw, off_nu, off_partial, off_final, off_score, ws_total;
 };
 
 // plan.cu
-ahakv_status make_plan(const ahakv_params* p, Plan* plan);
+// `obs_pos` (nullable, host, r ascending logical positions) places the observation rows; by default they are the
+// last r positions.
+ahakv_status make_plan(const ahakv_params* p, Plan* plan, const int64_t* obs_pos = nullptr);
 void count_launch(int n = 1);
 
 // Launchers.  Each returns AHAKV_OK or AHAKV_ERR_CUDA and queues work on `st` only.
@@ -52,12 +56,6 @@ ahakv_status launch_score_simt(const Plan& pl, const void* q, const void* k, flo
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
                              float2* partial, int* counters, int* status, cudaStream_t st);
 bool score_tc_available();
-// The tensor-core kernel that keeps the softmax numerators in tensor memory (score_res.cu): each key tile is
-// fetched, multiplied and exponentiated once.  `partial` holds one float per (row block, tile, row), `lfin` one
-// per (row block, row).  Takes the problems score_res_fits() accepts; the two-pass kernel takes the others.
-bool score_res_fits(const Plan& pl);
-ahakv_status launch_score_res(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
-                              float* partial, float* lfin, int* status, cudaStream_t st);
 ahakv_status launch_vnorm(const Plan& pl, const void* v, float* nu, cudaStream_t st);
 // `slots` partial scores per head (row blocks, or query heads when pooling by maximum) are combined here.
 ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,

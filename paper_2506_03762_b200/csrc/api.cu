@@ -2,7 +2,6 @@
 // layout and the order in which the kernels are queued.
 #include <atomic>
 #include <cmath>
-#include <cstdlib>
 #include <cstring>
 
 #include "ahakv_internal.cuh"
@@ -39,7 +38,7 @@ static bool resolve_strides(const int64_t in[3], long long out[3], long long hea
   return out[2] >= d;
 }
 
-ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
+ahakv_status make_plan(const ahakv_params* p, Plan* pl, const int64_t* obs_pos) {
   if (!p || !pl) return AHAKV_ERR_INVALID_ARG;
   if (p->batch < 1 || p->n_q_heads < 1 || p->n_kv_heads < 1 || p->n_q_heads % p->n_kv_heads != 0)
     return AHAKV_ERR_INVALID_ARG;
@@ -73,16 +72,21 @@ ahakv_status make_plan(const ahakv_params* p, Plan* pl) {
       !resolve_strides(p->v_stride, o.vs, o.Hkv, o.n, o.d, o.es))
     return AHAKV_ERR_INVALID_ARG;
 
-  for (int i = 0; i < kMaxRows; ++i) { o.rows.c[i] = 0.f; o.lambda[i] = 0.0; }
+  for (int i = 0; i < kMaxRows; ++i) { o.rows.c[i] = 0.f; o.lambda[i] = 0.0; o.last[i] = 0; }
+  const long long first_cached = p->n_total - p->n_ctx;      // logical position of cache row 0
   for (int i = 0; i < o.r; ++i) {
+    const long long pos = obs_pos ? obs_pos[i] : p->n_total - p->obs_window + i;
+    if (pos < first_cached || pos >= p->n_total || (i > 0 && obs_pos && pos <= obs_pos[i - 1])) return AHAKV_ERR_INVALID_ARG;
+    o.last[i] = (int)(pos - first_cached);
     double lam;
     if (p->scale_mode == AHAKV_SCALE_FIXED) lam = (double)p->scale;
-    else if (p->scale_mode == AHAKV_SCALE_ADAPTIVE_ROW)
-      lam = eq12((double)(p->n_total - p->obs_window + i + 1), (double)p->budget, p->head_dim);
+    else if (p->scale_mode == AHAKV_SCALE_ADAPTIVE_ROW) lam = eq12((double)(pos + 1), (double)p->budget, p->head_dim);
     else lam = eq12((double)p->n_total, (double)p->budget, p->head_dim);
     o.lambda[i] = lam;
     o.rows.c[i] = (float)(lam * 1.4426950408889634);
   }
+
+  o.n_eff = o.last[o.r - 1] + 1;
 
   // Tensor-core scoring: 16-bit inputs.  A row block stacks up to 128 / r query heads of one KV head (one TMA
   // box); when G is not a multiple of that, the last block of each KV head simply holds fewer heads.
@@ -137,18 +141,22 @@ static ahakv_status queue_raw_score(const Plan& pl, const void* q, const void* k
   float* final_off = at<float>(ws, pl.off_final);
   const bool prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0;
   float* nu = prior ? at<float>(ws, pl.off_nu) : nullptr;
-  static const bool two_pass_only = std::getenv("AHAKV_TWO_PASS_SCORING") != nullptr;   // measurement switch
-  if (pl.use_tc && !two_pass_only && score_res_fits(pl))   // the tensor-core kernels square the value rows on their way
-    rc = launch_score_res(pl, q, k, prior ? v : nullptr, s_raw, nu, reinterpret_cast<float*>(partial), final_off,
-                          at<int>(ws, pl.off_status), st);
-  else if (pl.use_tc)
-    rc = launch_score_tc(pl, q, k, prior ? v : nullptr, s_raw, nu, partial, at<int>(ws, pl.off_sync),
+  // The tensor-core kernel squares the value rows on its way, as long as its tiles cover all of them: when no
+  // observation row sees the last keys it skips their tiles, their raw score is zero and their value rows are
+  // squared by the streaming kernel.
+  const bool all_keys = pl.n_eff == pl.n;
+  const bool tc_prior = prior && pl.use_tc && all_keys;
+  if (pl.use_tc && !all_keys &&
+      cudaMemsetAsync(s_raw, 0, pl.off_nu - pl.off_sraw, st) != cudaSuccess)
+    return AHAKV_ERR_CUDA;
+  if (pl.use_tc)
+    rc = launch_score_tc(pl, q, k, tc_prior ? v : nullptr, s_raw, nu, partial, at<int>(ws, pl.off_sync),
                          at<int>(ws, pl.off_status), st);
   else
     rc = launch_score_simt(pl, q, k, s_raw, partial, final_off, st);
   if (rc) return rc;
   profile_mark(prof, 1, st);
-  if (prior && !pl.use_tc) {
+  if (prior && !tc_prior) {
     rc = launch_vnorm(pl, v, nu, st);
     if (rc) return rc;
   }
@@ -175,11 +183,11 @@ double ahakv_lambda(int64_t n_total, int32_t budget, int32_t head_dim) {
   return eq12((double)n_total, (double)budget, head_dim);
 }
 
-ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
-                         const float* score_prev, float* score, void* ws, size_t ws_bytes,
-                         ahakv_stream_t stream) {
+static ahakv_status score_impl(const ahakv_params* p, const int64_t* obs_pos, const void* q_obs, const void* k,
+                               const void* v, const float* score_prev, float* score, void* ws, size_t ws_bytes,
+                               cudaStream_t st) {
   Plan pl;
-  ahakv_status rc = make_plan(p, &pl);
+  ahakv_status rc = make_plan(p, &pl, obs_pos);
   if (rc) return rc;
   const bool prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0;
   if (!q_obs || !k || !score || (prior && !v)) return AHAKV_ERR_INVALID_ARG;
@@ -187,8 +195,7 @@ ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k
       (score_prev && !aligned16(score_prev)))
     return AHAKV_ERR_INVALID_ARG;
   if ((rc = check_ws(pl, ws, ws_bytes))) return rc;
-  const int prof = profile_begin_call((cudaStream_t)stream);
-  cudaStream_t st = (cudaStream_t)stream;
+  const int prof = profile_begin_call(st);
   if ((rc = queue_raw_score(pl, q_obs, k, v, ws, st, prof))) return rc;
   rc = launch_refine(pl, at<float>(ws, pl.off_sraw), prior ? at<float>(ws, pl.off_nu) : nullptr, score_prev, score,
                      score_slots(pl), st);
@@ -196,6 +203,67 @@ ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k
   profile_mark(prof, 4, st);   // no selection or compaction in this call
   profile_mark(prof, 5, st);
   return rc;
+}
+
+ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
+                         const float* score_prev, float* score, void* ws, size_t ws_bytes,
+                         ahakv_stream_t stream) {
+  return score_impl(p, nullptr, q_obs, k, v, score_prev, score, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+ahakv_status ahakv_score_rows(const ahakv_params* p, const int64_t* obs_pos, const void* q_obs, const void* k,
+                              const void* v, const float* score_prev, float* score, void* ws, size_t ws_bytes,
+                              ahakv_stream_t stream) {
+  if (!obs_pos) return AHAKV_ERR_INVALID_ARG;
+  return score_impl(p, obs_pos, q_obs, k, v, score_prev, score, ws, ws_bytes, (cudaStream_t)stream);
+}
+
+ahakv_status ahakv_score_full_causal(const ahakv_params* p, const void* q_all, const void* k, const void* v,
+                                     const float* score_prev, float* score, void* ws, size_t ws_bytes,
+                                     ahakv_stream_t stream) {
+  Plan full;
+  ahakv_status rc = make_plan(p, &full);      // validates everything but the query layout; sizes the workspace
+  if (rc) return rc;
+  if (full.group_max) return AHAKV_ERR_UNSUPPORTED;   // a maximum over heads of sums over passes is not a sum of maxima
+  const bool prior = (full.flags & AHAKV_FLAG_VALUE_PRIOR) != 0;
+  if (!q_all || !k || !score || (prior && !v)) return AHAKV_ERR_INVALID_ARG;
+  if (!aligned16(q_all) || !aligned16(k) || (v && !aligned16(v)) || !aligned16(score) ||
+      (score_prev && !aligned16(score_prev)))
+    return AHAKV_ERR_INVALID_ARG;
+  if ((rc = check_ws(full, ws, ws_bytes))) return rc;
+  cudaStream_t st = (cudaStream_t)stream;
+  // q_all holds a query for every cached row: [B, Hq, n, d] unless strides say otherwise
+  ahakv_params pc = *p;
+  if (p->q_stride[0] == 0 && p->q_stride[1] == 0 && p->q_stride[2] == 0) {
+    pc.q_stride[2] = p->head_dim;
+    pc.q_stride[1] = (int64_t)p->n_ctx * p->head_dim;
+    pc.q_stride[0] = (int64_t)p->n_q_heads * p->n_ctx * p->head_dim;
+  }
+  pc.flags = p->flags & ~(uint32_t)AHAKV_FLAG_VALUE_PRIOR;     // the prior multiplies the finished sum, once
+  float* acc = at<float>(ws, full.off_score);                  // running sum over the passes, [B, Hkv, n]
+  const int R = p->obs_window, n = p->n_ctx;
+  const long long first_cached = p->n_total - p->n_ctx;
+  int64_t pos[kMaxRows];
+  for (int c0 = 0; c0 < n; c0 += R) {
+    const int rows = n - c0 < R ? n - c0 : R;
+    pc.obs_window = rows;
+    for (int i = 0; i < rows; ++i) pos[i] = first_cached + c0 + i;
+    Plan pl;
+    if ((rc = make_plan(&pc, &pl, pos))) return rc;
+    if (pl.off_score > full.off_score) return AHAKV_ERR_WORKSPACE;   // cannot happen: fewer rows never need more room
+    const char* qc = (const char*)q_all + (size_t)c0 * pl.qs[2] * pl.es;
+    if ((rc = queue_raw_score(pl, qc, k, nullptr, ws, st, -1))) return rc;
+    if ((rc = launch_refine(pl, at<float>(ws, pl.off_sraw), nullptr, c0 == 0 ? nullptr : acc, acc, score_slots(pl), st)))
+      return rc;
+  }
+  float* nu = nullptr;
+  if (prior) {
+    nu = at<float>(ws, full.off_nu);
+    if ((rc = launch_vnorm(full, v, nu, st))) return rc;
+  }
+  Plan one = full;
+  one.group_max = 0;
+  return launch_refine(one, acc, nu, score_prev, score, 1, st);
 }
 
 ahakv_status ahakv_select(const ahakv_params* p, const float* score, int32_t* kept_idx, void* ws,

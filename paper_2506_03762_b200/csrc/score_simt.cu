@@ -50,9 +50,10 @@ __device__ __forceinline__ void load_key(const T* __restrict__ k, const Shape& p
 // The accumulator type of the logits: double for float32 inputs, float for 16-bit ones.
 template <typename T> using Acc = typename std::conditional<std::is_same<T, float>::value, double, float>::type;
 
-// lambda_i log2(e) per observation row in the accumulator's type.
+// Per observation row: lambda_i log2(e) in the accumulator's type, and the last cache row it may see.
 template <typename A> struct RowScaleOf {
   A c[kMaxRows];
+  int last[kMaxRows];
 };
 
 template <int D, typename A>
@@ -91,7 +92,7 @@ __global__ void __launch_bounds__(kThreads) simt_row_stats(const T* __restrict__
   __syncthreads();
   for (int s = 0; s < pl.R; ++s) {
     const int i = s % pl.r;
-    const bool vis = valid && j <= pl.n - pl.r + i;
+    const bool vis = valid && j <= cs.last[i];
     const A x = vis ? dot_row<D, A>(qsm + s * D, kreg) * cs.c[i] : (A)-INFINITY;
     float m = (float)x;                                         // the shift is an FP32 number on either path
 #pragma unroll
@@ -158,7 +159,7 @@ __global__ void __launch_bounds__(kThreads) simt_column_sums(const T* __restrict
       best = fmaxf(best, acc);
       acc = 0.f;
     }
-    if (j <= pl.n - pl.r + i)
+    if (j <= cs.last[i])
       acc = fmaf(fast_exp2((float)fma(dot_row<D, A>(qsm + s * D, kreg), cs.c[i], -(A)st[s].x)), st[s].y, acc);
   }
   s_raw[(size_t)unit * pl.n + j] = pl.group_max ? fmaxf(best, acc) : acc;
@@ -168,7 +169,10 @@ template <typename T, int D>
 ahakv_status run(const Plan& pl, const void* q, const void* k, float* s_raw, float2* partial, float* final_off,
                  cudaStream_t st) {
   RowScaleOf<Acc<T>> cs;
-  for (int i = 0; i < kMaxRows; ++i) cs.c[i] = i < pl.r ? (Acc<T>)(pl.lambda[i] * 1.4426950408889634) : (Acc<T>)0;
+  for (int i = 0; i < kMaxRows; ++i) {
+    cs.c[i] = i < pl.r ? (Acc<T>)(pl.lambda[i] * 1.4426950408889634) : (Acc<T>)0;
+    cs.last[i] = pl.last[i];
+  }
   const size_t smem1 = (size_t)pl.R * D * sizeof(float) + (size_t)(kThreads / 32) * pl.R * sizeof(float2);
   const size_t smem2 = (size_t)pl.R * D * sizeof(float) + (size_t)pl.R * sizeof(float2);
   if (cudaFuncSetAttribute(simt_row_stats<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1) != cudaSuccess ||

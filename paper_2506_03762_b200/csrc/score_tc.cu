@@ -87,6 +87,8 @@ struct TcArgs {
   float log2G;
   float c[kMaxRows];     // lambda_i log2(e) per observation row
   float cs[128];         // the same per stacked row of a row block (r <= 128 only)
+  int last[kMaxRows];    // per observation row: the last key it may see
+  int min_last;          // the smallest of them: tiles that end at or before it are masked for no row
   float* partial;    // [unit][run][128]: log2 of a row's sum of 2^{c w} over the run's keys
   float* s_raw;      // [unit][n]
   float* nu;         // [B * Hkv][n]
@@ -112,7 +114,7 @@ struct Shared {
   int mrg[kMergeRing];                      // run, or kSegEnd
   float c[kMaxRows];            // lambda_i * log2(e) per observation row
   float cs2[2][128];            // c per stacked row, by row block parity (r > 128 has two kinds of block)
-  int vis_off[2][128];          // per stacked row: n - r + its observation row = the last key it may see
+  int vis_off[2][128];          // per stacked row: the last key its observation row may see
   float2 p1_part[2][3][128];    // pass 1: statistics of the three groups that do not publish
   float p2_part[2][3][128];     // pass 2: partial column sums of the three groups that do not store
 };
@@ -602,7 +604,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
     if (pass == 0) {
       const int i = obs_row(a, u, s);
       const float c = sh->c[i < a.r ? i : 0];
-      const int last = a.n - a.r + i;                       // last visible key of this row
+      const int last = a.last[i < kMaxRows ? i : 0];        // last visible key of this row
       float M = -INFINITY, Z = 0.f;
       for (int t = 0; t < rn.cnt; ++t, ++tc) {
         if (gone) continue;
@@ -610,7 +612,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
         if (!mbar_wait(&bars->acc_full[acc], aph, a.status)) { gone = true; continue; }
         tc_fence_after();
         const int j0 = (rn.blk0 + t) * kKeyTile + 32 * g;
-        const bool full = (rn.blk0 + t) * kKeyTile + kKeyTile - 1 <= a.n - a.r;   // no key of the tile is masked
+        const bool full = (rn.blk0 + t) * kKeyTile + kKeyTile - 1 <= a.min_last;   // no key of the tile is masked
         uint32_t ra[32];
         tmem_ld32_issue(lane_base + (uint32_t)(acc * 128 + 32 * g), ra);
         tmem_ld_wait(ra);
@@ -652,7 +654,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
         if (!gone && !mbar_wait(&bars->acc_full[acc], aph, a.status)) gone = true;
         if (!gone) {
           tc_fence_after();
-          const bool full = j0 + kKeyTile - 1 <= a.n - a.r;
+          const bool full = j0 + kKeyTile - 1 <= a.min_last;
           const uint32_t taddr = lane_base + (uint32_t)(acc * 128);
           if (full && fast) {
             void* ae = &bars->acc_empty[acc];
@@ -803,8 +805,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   for (int t = threadIdx.x; t < 128; t += kThreads) {
     sh->cs2[0][t] = a.r <= 128 ? a.c[t % a.r] : a.c[t];
     sh->cs2[1][t] = a.r <= 128 ? a.c[t % a.r] : a.c[128 + t];
-    sh->vis_off[0][t] = a.n - a.r + (a.r <= 128 ? t % a.r : t);
-    sh->vis_off[1][t] = a.n - a.r + (a.r <= 128 ? t % a.r : 128 + t);
+    sh->vis_off[0][t] = a.last[a.r <= 128 ? t % a.r : t];
+    sh->vis_off[1][t] = a.last[a.r <= 128 ? t % a.r : 128 + t];
   }
   {
     // every 16-byte chunk of the constant tile reads (kFold, kFold, kFold, 0, 0, 0, 0, 0); it meets the
@@ -898,12 +900,15 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   const int units = pl.B * pl.Hkv * pl.n_rb;
   TcArgs a;
   a.n = pl.n; a.r = pl.r; a.G = pl.G; a.Hkv = pl.Hkv; a.n_rb = pl.n_rb; a.hb = pl.heads_per_rb;
-  a.n_blk = pl.n_blk; a.D = pl.d;
+  a.n_blk = (pl.n_eff + kKeyTile - 1) / kKeyTile;   // tiles beyond are seen by no row
+  a.D = pl.d;
+  for (int i = 0; i < kMaxRows; ++i) a.last[i] = pl.last[i];
+  a.min_last = pl.last[0];
   // Runs of 8 tiles; shorter ones (4, 2, 1) only as far as it takes to give three SMs in four a run.  Every run
   // boundary drains the pipeline, which costs more than a few idle SMs on a small problem.
   a.CH = 8;
-  while (a.CH > 1 && (long long)units * ((pl.n_blk + a.CH - 1) / a.CH) * 4 < (long long)n_sm * 3) a.CH >>= 1;
-  a.rpu = (pl.n_blk + a.CH - 1) / a.CH;
+  while (a.CH > 1 && (long long)units * ((a.n_blk + a.CH - 1) / a.CH) * 4 < (long long)n_sm * 3) a.CH >>= 1;
+  a.rpu = (a.n_blk + a.CH - 1) / a.CH;
   a.n_runs = units * a.rpu;
   const int grid = a.n_runs < n_sm ? a.n_runs : n_sm;
   a.bf16 = pl.dtype == AHAKV_BF16;
