@@ -120,6 +120,15 @@ ahakv_status ahakv_score_full_causal(const ahakv_params* p, const void* q_all, c
                                      const float* score_prev, float* score, void* ws, size_t ws_bytes,
                                      ahakv_stream_t stream);
 
+/* Row entropy of the scaled softmax (Section 4.2, Eq. 6): H_i = - sum_j a_ij ln a_ij (natural log) for every
+ * observation row of every query head, with a_ij exactly as in ahakv_score (mask, lambda from scale_mode).  A
+ * diagnostic: Eq. 10 predicts E[H_i] = ln i - lambda^2 d / 2, and Eq. 12 picks lambda so that this is ln(budget).
+ * entropy: [B,Hq,r] float32 out.  ws: ahakv_entropy_workspace_bytes(p) bytes, 256-byte aligned (not the scoring
+ * workspace).  Runs on the FP32 pipes (double for float32 inputs); it is not part of the eviction path. */
+size_t ahakv_entropy_workspace_bytes(const ahakv_params* p);
+ahakv_status ahakv_row_entropy(const ahakv_params* p, const void* q_obs, const void* k, float* entropy, void* ws,
+                               size_t ws_bytes, ahakv_stream_t stream);
+
 /* Selection (Algorithm 1: S^r = recent B_r tokens, S^s = TopK(F, B_s), S = S^s U S^r).
  * Keeps rows [n - B_r, n) and the B_s = budget - B_r highest-scoring rows of [0, n - B_r);
  * equal scores are taken lowest index first; the result is ascending.  n <= budget keeps all rows.

@@ -85,6 +85,8 @@ SIGNATURES = {
     "ahakv_score": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_score_rows": (ctypes.c_int, [_PP, ctypes.POINTER(ctypes.c_int64), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_score_full_causal": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_entropy_workspace_bytes": (_sz, [_PP]),
+    "ahakv_row_entropy": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_select": (ctypes.c_int, [_PP, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_compact": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_evict": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -187,6 +189,20 @@ def ahakv_score_full_causal(p: Params, q_all, k, v, score_prev, score, ws, ws_by
     if check:
         _raise(st, "ahakv_score_full_causal")
     return st
+
+
+def ahakv_row_entropy(p: Params, q_obs, k, entropy=None, stream=None):
+    """Eq. 6 entropy [B,Hq,r] (float32) of every observation row; allocates its scratch and, if not given, the output."""
+    cp = p.c()
+    nbytes = int(lib().ahakv_entropy_workspace_bytes(ctypes.byref(cp)))
+    if nbytes == 0:
+        raise AhakvError(ERR_INVALID_ARG, "ahakv_entropy_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=k.device)
+    if entropy is None:
+        entropy = torch.empty((p.batch, p.n_q_heads, p.obs_window), dtype=torch.float32, device=k.device)
+    _raise(lib().ahakv_row_entropy(ctypes.byref(cp), _ptr(q_obs), _ptr(k), _ptr(entropy), _ptr(ws), nbytes,
+                                   _stream(stream)), "ahakv_row_entropy")
+    return entropy
 
 
 def ahakv_static_workspace_bytes() -> int:

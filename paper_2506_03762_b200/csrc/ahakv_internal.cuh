@@ -56,6 +56,9 @@ ahakv_status launch_score_simt(const Plan& pl, const void* q, const void* k, flo
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
                              float2* partial, int* counters, int* status, cudaStream_t st);
 bool score_tc_available();
+// Row entropy of the SG-softmax (entropy.cu): out [B, Hq, r]; `scratch` of entropy_scratch_bytes().
+size_t entropy_scratch_bytes(const Plan& pl);
+ahakv_status launch_entropy(const Plan& pl, const void* q, const void* k, void* scratch, float* out, cudaStream_t st);
 ahakv_status launch_vnorm(const Plan& pl, const void* v, float* nu, cudaStream_t st);
 // `slots` partial scores per head (row blocks, or query heads when pooling by maximum) are combined here.
 ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,

@@ -266,6 +266,23 @@ ahakv_status ahakv_score_full_causal(const ahakv_params* p, const void* q_all, c
   return launch_refine(one, acc, nu, score_prev, score, 1, st);
 }
 
+size_t ahakv_entropy_workspace_bytes(const ahakv_params* p) {
+  Plan pl;
+  if (make_plan(p, &pl) != AHAKV_OK) return 0;
+  return entropy_scratch_bytes(pl);
+}
+
+ahakv_status ahakv_row_entropy(const ahakv_params* p, const void* q_obs, const void* k, float* entropy, void* ws,
+                               size_t ws_bytes, ahakv_stream_t stream) {
+  Plan pl;
+  ahakv_status rc = make_plan(p, &pl);
+  if (rc) return rc;
+  if (!q_obs || !k || !entropy || !aligned16(q_obs) || !aligned16(k) || ((uintptr_t)entropy & 3))
+    return AHAKV_ERR_INVALID_ARG;
+  if (!ws || ((uintptr_t)ws & 255) != 0 || ws_bytes < entropy_scratch_bytes(pl)) return AHAKV_ERR_WORKSPACE;
+  return launch_entropy(pl, q_obs, k, ws, entropy, (cudaStream_t)stream);
+}
+
 ahakv_status ahakv_select(const ahakv_params* p, const float* score, int32_t* kept_idx, void* ws,
                           size_t ws_bytes, ahakv_stream_t stream) {
   Plan pl;
