@@ -120,6 +120,24 @@ ahakv_status ahakv_score_full_causal(const ahakv_params* p, const void* q_all, c
                                      const float* score_prev, float* score, void* ws, size_t ws_bytes,
                                      ahakv_stream_t stream);
 
+/* One generation step of the score (Algorithm 1, Generation: A = q_t K^T, F_t = SGsoftmax(A) + F_{t-1}): the one
+ * new query of every head against the n cached keys (the new token's own key is row n - 1), pooled over the
+ * query heads of each KV head, plus score_prev (nullable; 0 for the new row).  p->obs_window must be 1.  A
+ * kernel of its own: K is read once with 16-byte loads, the G x n logits stay in shared memory, no scratch
+ * memory is needed.  It takes G <= 8 (or 12, 16) query heads per KV head and G * n <= 40960 logits, which covers
+ * caches held at their budget; larger problems and AHAKV_FLAG_VALUE_PRIOR (Algorithm 1's generation phase has
+ * no value prior) get AHAKV_ERR_UNSUPPORTED: use ahakv_score with obs_window 1 for those.
+ * q_t: [B,Hq,1,d].  score_prev, score: [B,Hkv,n] float32; they may be the same buffer. */
+ahakv_status ahakv_score_step(const ahakv_params* p, const void* q_t, const void* k, const float* score_prev,
+                              float* score, ahakv_stream_t stream);
+
+/* Compaction in place (Algorithm 1, Generation: K <- K_S, V <- V_S before the next token): rows kept_idx[t] of k,
+ * v (and of score, nullable, [B,Hkv,n]) move to rows t; rows from n_keep on are left as they are.  kept_idx is
+ * ascending, so rows before the first evicted index are not touched and only the rest is moved.  One CTA per
+ * (sequence, KV head), batches staged in shared memory.  The exception to "outputs must not alias inputs". */
+ahakv_status ahakv_compact_inplace(const ahakv_params* p, void* k, void* v, float* score, const int32_t* kept_idx,
+                                   ahakv_stream_t stream);
+
 /* Row entropy of the scaled softmax (Section 4.2, Eq. 6): H_i = - sum_j a_ij ln a_ij (natural log) for every
  * observation row of every query head, with a_ij exactly as in ahakv_score (mask, lambda from scale_mode).  A
  * diagnostic: Eq. 10 predicts E[H_i] = ln i - lambda^2 d / 2, and Eq. 12 picks lambda so that this is ln(budget).
@@ -132,7 +150,8 @@ ahakv_status ahakv_row_entropy(const ahakv_params* p, const void* q_obs, const v
 /* Selection (Algorithm 1: S^r = recent B_r tokens, S^s = TopK(F, B_s), S = S^s U S^r).
  * Keeps rows [n - B_r, n) and the B_s = budget - B_r highest-scoring rows of [0, n - B_r);
  * equal scores are taken lowest index first; the result is ascending.  n <= budget keeps all rows.
- * score: [B,Hkv,n] float32 in.  kept_idx: [B,Hkv,n_keep] int32 out. */
+ * score: [B,Hkv,n] float32 in.  kept_idx: [B,Hkv,n_keep] int32 out.  ws and ws_bytes are not used (selection
+ * works in shared memory) and may be NULL and 0. */
 ahakv_status ahakv_select(const ahakv_params* p, const float* score, int32_t* kept_idx, void* ws,
                           size_t ws_bytes, ahakv_stream_t stream);
 
@@ -188,10 +207,12 @@ const char* ahakv_stage_name(int stage);
  *  - All calls on a device share the one array, which keeps whatever the last call left in it.  The call
  *    resets what has to start clean, so calls in sequence are independent; two calls that overlap on the
  *    GPU (different streams) race on the array and must be serialised by the caller.
- *  - ahakv_last_device_status cannot be asked about this scratch; a device-side timeout leaves the output
- *    undefined, exactly as in ahakv_score. */
+ *  - ahakv_static_last_device_status(stream) is ahakv_last_device_status for this scratch (it synchronises
+ *    `stream`): after a device-side timeout the output is undefined, exactly as in ahakv_score.
+ * Parameters are judged exactly as ahakv_score judges them (same status codes). */
 #define AHAKV_STATIC_WS_BYTES (8u << 20)
 size_t ahakv_static_workspace_bytes(void);
+ahakv_status ahakv_static_last_device_status(ahakv_stream_t stream);
 ahakv_status ahakv_score_static(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
                                 const float* score_prev, float* score, ahakv_stream_t stream);
 

@@ -85,6 +85,8 @@ SIGNATURES = {
     "ahakv_score": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_score_rows": (ctypes.c_int, [_PP, ctypes.POINTER(ctypes.c_int64), _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_score_full_causal": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_score_step": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp]),
+    "ahakv_compact_inplace": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_entropy_workspace_bytes": (_sz, [_PP]),
     "ahakv_row_entropy": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_select": (ctypes.c_int, [_PP, _vp, _vp, _vp, _sz, _vp]),
@@ -92,6 +94,7 @@ SIGNATURES = {
     "ahakv_evict": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_score_static": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_static_workspace_bytes": (_sz, []),
+    "ahakv_static_last_device_status": (ctypes.c_int, [_vp]),
     "ahakv_last_device_status": (ctypes.c_int, [_vp, _vp]),
     "ahakv_launch_count": (ctypes.c_int64, []),
     "ahakv_profile_enable": (ctypes.c_int, [ctypes.c_int]),
@@ -191,6 +194,22 @@ def ahakv_score_full_causal(p: Params, q_all, k, v, score_prev, score, ws, ws_by
     return st
 
 
+def ahakv_score_step(p: Params, q_t, k, score_prev, score, stream=None, check: bool = True) -> int:
+    cp = p.c()
+    st = lib().ahakv_score_step(ctypes.byref(cp), _ptr(q_t), _ptr(k), _ptr(score_prev), _ptr(score), _stream(stream))
+    if check:
+        _raise(st, "ahakv_score_step")
+    return st
+
+
+def ahakv_compact_inplace(p: Params, k, v, score, kept_idx, stream=None, check: bool = True) -> int:
+    cp = p.c()
+    st = lib().ahakv_compact_inplace(ctypes.byref(cp), _ptr(k), _ptr(v), _ptr(score), _ptr(kept_idx), _stream(stream))
+    if check:
+        _raise(st, "ahakv_compact_inplace")
+    return st
+
+
 def ahakv_row_entropy(p: Params, q_obs, k, entropy=None, stream=None):
     """Eq. 6 entropy [B,Hq,r] (float32) of every observation row; allocates its scratch and, if not given, the output."""
     cp = p.c()
@@ -209,6 +228,10 @@ def ahakv_static_workspace_bytes() -> int:
     return int(lib().ahakv_static_workspace_bytes())
 
 
+def ahakv_static_last_device_status(stream=None) -> int:
+    return int(lib().ahakv_static_last_device_status(_stream(stream)))
+
+
 def ahakv_score_static(p: Params, q_obs, k, v, score_prev, score, stream=None, check: bool = True) -> int:
     """``ahakv_score`` on the library's own fixed scratch array: no workspace argument, no allocation."""
     cp = p.c()
@@ -219,10 +242,10 @@ def ahakv_score_static(p: Params, q_obs, k, v, score_prev, score, stream=None, c
     return st
 
 
-def ahakv_select(p: Params, score, kept_idx, ws, ws_bytes: int | None = None, stream=None,
+def ahakv_select(p: Params, score, kept_idx, ws=None, ws_bytes: int | None = None, stream=None,
                  check: bool = True) -> int:
     cp = p.c()
-    nbytes = ws.numel() * ws.element_size() if ws_bytes is None else ws_bytes
+    nbytes = (0 if ws is None else ws.numel() * ws.element_size()) if ws_bytes is None else ws_bytes
     st = lib().ahakv_select(ctypes.byref(cp), _ptr(score), _ptr(kept_idx), _ptr(ws), nbytes, _stream(stream))
     if check:
         _raise(st, "ahakv_select")

@@ -56,6 +56,13 @@ ahakv_status launch_score_simt(const Plan& pl, const void* q, const void* k, flo
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
                              float2* partial, int* counters, int* status, cudaStream_t st);
 bool score_tc_available();
+// The generation phase one token at a time (decode.cu): the score update of one new query per head without
+// scratch memory, and compaction in place.
+bool step_score_fits(const Plan& pl);
+ahakv_status launch_step_score(const Plan& pl, const void* q, const void* k, const float* prev, float* score,
+                               cudaStream_t st);
+ahakv_status launch_compact_inplace(const Plan& pl, void* k, void* v, float* score, const int32_t* kept_idx,
+                                    cudaStream_t st);
 // Row entropy of the SG-softmax (entropy.cu): out [B, Hq, r]; `scratch` of entropy_scratch_bytes().
 size_t entropy_scratch_bytes(const Plan& pl);
 ahakv_status launch_entropy(const Plan& pl, const void* q, const void* k, void* scratch, float* out, cudaStream_t st);

@@ -266,6 +266,30 @@ ahakv_status ahakv_score_full_causal(const ahakv_params* p, const void* q_all, c
   return launch_refine(one, acc, nu, score_prev, score, 1, st);
 }
 
+ahakv_status ahakv_score_step(const ahakv_params* p, const void* q_t, const void* k, const float* score_prev,
+                              float* score, ahakv_stream_t stream) {
+  Plan pl;
+  ahakv_status rc = make_plan(p, &pl);
+  if (rc) return rc;
+  if (pl.r != 1) return AHAKV_ERR_INVALID_ARG;
+  if (!q_t || !k || !score || !aligned16(q_t) || !aligned16(k) || !aligned16(score) ||
+      (score_prev && !aligned16(score_prev)))
+    return AHAKV_ERR_INVALID_ARG;
+  if ((pl.flags & AHAKV_FLAG_VALUE_PRIOR) || !step_score_fits(pl)) return AHAKV_ERR_UNSUPPORTED;
+  return launch_step_score(pl, q_t, k, score_prev, score, (cudaStream_t)stream);
+}
+
+ahakv_status ahakv_compact_inplace(const ahakv_params* p, void* k, void* v, float* score, const int32_t* kept_idx,
+                                   ahakv_stream_t stream) {
+  Plan pl;
+  ahakv_status rc = make_plan(p, &pl);
+  if (rc) return rc;
+  if (!k || !v || !kept_idx || !aligned16(k) || !aligned16(v) || ((uintptr_t)kept_idx & 3) ||
+      (score && ((uintptr_t)score & 3)))
+    return AHAKV_ERR_INVALID_ARG;
+  return launch_compact_inplace(pl, k, v, score, kept_idx, (cudaStream_t)stream);
+}
+
 size_t ahakv_entropy_workspace_bytes(const ahakv_params* p) {
   Plan pl;
   if (make_plan(p, &pl) != AHAKV_OK) return 0;
@@ -289,7 +313,7 @@ ahakv_status ahakv_select(const ahakv_params* p, const float* score, int32_t* ke
   ahakv_status rc = make_plan(p, &pl);
   if (rc) return rc;
   if (!score || !kept_idx || !aligned16(score) || ((uintptr_t)kept_idx & 3)) return AHAKV_ERR_INVALID_ARG;
-  if ((rc = check_ws(pl, ws, ws_bytes))) return rc;
+  (void)ws; (void)ws_bytes;                    // selection works in shared memory: no scratch is needed
   return launch_select(pl, score, kept_idx, (cudaStream_t)stream);
 }
 

@@ -1,0 +1,250 @@
+// The generation phase one token at a time (Algorithm 1, Generation: A = q_t K^T, F_t = SGsoftmax(A) + F_{t-1},
+// then S = TopK(F_t, B_s) U recent B_r and K <- K_S, V <- V_S before the next token).
+//
+// step_score_kernel: one CTA per (sequence, KV head).  The G query rows of the group (one new query per head)
+//   against the n cached keys is a matrix-vector product, bound by reading K once: half a warp (or a quarter,
+//   or a whole one, by row size) reads one key row with 16-byte loads, every lane keeps its slice of the G
+//   queries in registers, and the partial dot products meet by shuffle.  The G x n logits stay in shared memory;
+//   row maxima and sums are block reductions in a fixed order; the new score is written in one more sweep.
+//   No scratch memory, no second read of K.
+//
+// compact_inplace_kernel: one CTA per (sequence, KV head).  kept_idx is ascending, so row t of the result comes
+//   from row kept_idx[t] >= t: rows before the first evicted index do not move at all, and the others move in
+//   batches through shared memory (all loads of a batch, a barrier, all its stores), so no row is overwritten
+//   before it has been read.
+#include <type_traits>
+
+#include "ahakv_internal.cuh"
+
+namespace ahakv {
+namespace {
+
+constexpr int kStepThreads = 256;
+constexpr int kStepMaxG = 16;                  // query heads per KV head the step kernel takes
+constexpr size_t kStepMaxLogitBytes = 160 * 1024;   // 40960 logits
+
+template <typename T> using Acc = typename std::conditional<std::is_same<T, float>::value, double, float>::type;
+
+// Block-wide reduction in a fixed order: warp shuffles, then the warps' results in warp order.
+template <bool kMax>
+__device__ __forceinline__ float block_reduce(float x, float* red) {
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    const float y = __shfl_xor_sync(0xffffffffu, x, o);
+    x = kMax ? fmaxf(x, y) : x + y;
+  }
+  __syncthreads();                              // `red` may still be read from the last reduction
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
+  __syncthreads();
+  float r = red[0];
+  for (int w = 1; w < kStepThreads / 32; ++w) r = kMax ? fmaxf(r, red[w]) : r + red[w];
+  return r;
+}
+
+// LANES threads share a key row (16 bytes each); kG query heads.
+template <typename T, int D, int kG>
+__global__ void __launch_bounds__(kStepThreads) step_score_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                                  const float* __restrict__ prev,
+                                                                  float* __restrict__ score, const Shape pl,
+                                                                  const double c_row) {
+  using A = Acc<T>;
+  constexpr int V = Vec16<T>::N, LANES = D / V, KEYS_PER_WARP = 32 / LANES;
+  extern __shared__ __align__(16) float logit[];                 // [kG][n]
+  __shared__ float red[kStepThreads / 32];
+  const int unit = blockIdx.x, b = unit / pl.Hkv, h = unit % pl.Hkv, n = pl.n;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, sub = lane % LANES, which = lane / LANES;
+  const A c = (A)c_row;
+
+  // this lane's slice of each of the group's queries
+  float qreg[kG][V];
+#pragma unroll
+  for (int g = 0; g < kG; ++g) {
+    const T* row = q + (long long)b * pl.qs[0] + (long long)(h * pl.G + g) * pl.qs[1];
+    Vec16<T>::widen(*reinterpret_cast<const uint4*>(row + sub * V), qreg[g]);
+  }
+  const T* kbase = k + (long long)b * pl.ks[0] + (long long)h * pl.ks[1];
+  constexpr int kUnroll = 4;                                     // key rows in flight per lane
+  const int stride = (kStepThreads / 32) * KEYS_PER_WARP;
+  for (int j0 = warp * KEYS_PER_WARP + which; j0 - which < n; j0 += stride * kUnroll) {
+    uint4 raw[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int j = j0 + u * stride;
+      raw[u] = j < n ? *reinterpret_cast<const uint4*>(kbase + (long long)j * pl.ks[2] + sub * V) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int j = j0 + u * stride;
+      float kv[V];
+      Vec16<T>::widen(raw[u], kv);
+#pragma unroll
+      for (int g = 0; g < kG; ++g) {
+        A acc = 0;
+#pragma unroll
+        for (int e = 0; e < V; ++e) acc = fma((A)qreg[g][e], (A)kv[e], acc);
+#pragma unroll
+        for (int o = LANES / 2; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (sub == 0 && j < n) logit[g * n + j] = (float)(acc * c);    // log2 units
+      }
+    }
+  }
+  __syncthreads();
+
+  // per query head: shift and normaliser, then 2^{x - M} / (G Z) in place
+  const float inv_g = pl.group_max ? 1.f : 1.f / (float)kG;
+  for (int g = 0; g < kG; ++g) {
+    float* x = logit + g * n;
+    float m = -INFINITY;
+    for (int j = threadIdx.x; j < n; j += kStepThreads) m = fmaxf(m, x[j]);
+    const float M = block_reduce<true>(m, red);
+    float z = 0.f;
+    for (int j = threadIdx.x; j < n; j += kStepThreads) {
+      const float e = fast_exp2(x[j] - M);
+      x[j] = e;
+      z += e;
+    }
+    const float Z = block_reduce<false>(z, red);
+    const float w = inv_g / Z;
+    for (int j = threadIdx.x; j < n; j += kStepThreads) x[j] *= w;
+  }
+  __syncthreads();
+  for (int j = threadIdx.x; j < n; j += kStepThreads) {
+    float s = logit[j];
+#pragma unroll
+    for (int g = 1; g < kG; ++g) s = pl.group_max ? fmaxf(s, logit[g * n + j]) : s + logit[g * n + j];
+    if (prev) s = __fadd_rn(s, prev[(size_t)unit * n + j]);
+    score[(size_t)unit * n + j] = s;
+  }
+}
+
+template <typename T, int D, int kG>
+ahakv_status launch_step_as(const Plan& pl, const void* q, const void* k, const float* prev, float* score,
+                            cudaStream_t st) {
+  const size_t smem = (size_t)kG * pl.n * sizeof(float);
+  constexpr int kMaxDevices = 64;
+  static size_t configured[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AHAKV_ERR_CUDA;
+  if (smem > 40 * 1024 && configured[dev] < kStepMaxLogitBytes) {
+    if (cudaFuncSetAttribute(step_score_kernel<T, D, kG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kStepMaxLogitBytes) != cudaSuccess)
+      return AHAKV_ERR_CUDA;
+    configured[dev] = kStepMaxLogitBytes;
+  }
+  const Shape& shape = pl;
+  step_score_kernel<T, D, kG><<<pl.B * pl.Hkv, kStepThreads, smem, st>>>((const T*)q, (const T*)k, prev, score, shape,
+                                                                      pl.lambda[0] * 1.4426950408889634);
+  count_launch();
+  return cuda_ok(cudaGetLastError());
+}
+
+template <typename T, int D>
+ahakv_status launch_step_g(const Plan& pl, const void* q, const void* k, const float* prev, float* score, cudaStream_t st) {
+  switch (pl.G) {
+    case 1: return launch_step_as<T, D, 1>(pl, q, k, prev, score, st);
+    case 2: return launch_step_as<T, D, 2>(pl, q, k, prev, score, st);
+    case 3: return launch_step_as<T, D, 3>(pl, q, k, prev, score, st);
+    case 4: return launch_step_as<T, D, 4>(pl, q, k, prev, score, st);
+    case 5: return launch_step_as<T, D, 5>(pl, q, k, prev, score, st);
+    case 6: return launch_step_as<T, D, 6>(pl, q, k, prev, score, st);
+    case 7: return launch_step_as<T, D, 7>(pl, q, k, prev, score, st);
+    case 8: return launch_step_as<T, D, 8>(pl, q, k, prev, score, st);
+    case 12: return launch_step_as<T, D, 12>(pl, q, k, prev, score, st);
+    case 16: return launch_step_as<T, D, 16>(pl, q, k, prev, score, st);
+    default: return AHAKV_ERR_UNSUPPORTED;
+  }
+}
+
+// ---- in-place compaction ------------------------------------------------------------------------------------------
+constexpr int kMoveThreads = 512;
+constexpr int kMoveBatchBytes = 96 * 1024;      // staged per batch: K rows, V rows (and scores)
+
+__global__ void __launch_bounds__(kMoveThreads) compact_inplace_kernel(char* __restrict__ k, char* __restrict__ v,
+                                                                       float* __restrict__ score,
+                                                                       const int32_t* __restrict__ kept, const Shape pl,
+                                                                       const int rows_per_batch) {
+  extern __shared__ __align__(16) char stage[];
+  __shared__ int first_moved;
+  const int unit = blockIdx.x, n_keep = pl.n_keep;
+  const long long b = unit / pl.Hkv, h = unit % pl.Hkv;
+  const int32_t* idx = kept + (size_t)unit * n_keep;
+  const int row_bytes = pl.d * pl.es, lanes = row_bytes / 16;
+  char* kb = k + (b * pl.ks[0] + h * pl.ks[1]) * pl.es;
+  char* vb = v + (b * pl.vs[0] + h * pl.vs[1]) * pl.es;
+  const long long ktok = pl.ks[2] * pl.es, vtok = pl.vs[2] * pl.es;
+  float* sc = score ? score + (size_t)unit * pl.n : nullptr;
+
+  // rows before the first evicted index stay where they are
+  if (threadIdx.x == 0) first_moved = n_keep;
+  __syncthreads();
+  for (int t = threadIdx.x; t < n_keep; t += kMoveThreads)
+    if (idx[t] != t) { atomicMin(&first_moved, t); break; }       // ascending indices: the thread's first is its smallest
+  __syncthreads();
+  const int t_begin = first_moved;
+
+  uint4* ks = reinterpret_cast<uint4*>(stage);
+  uint4* vs = ks + (size_t)rows_per_batch * lanes;
+  float* ss = reinterpret_cast<float*>(vs + (size_t)rows_per_batch * lanes);
+  for (int t0 = t_begin; t0 < n_keep; t0 += rows_per_batch) {
+    const int rows = min(rows_per_batch, n_keep - t0), chunks = rows * lanes;
+    for (int c = threadIdx.x; c < chunks; c += kMoveThreads) {
+      const int t = c / lanes, sub = c % lanes;
+      const long long j = idx[t0 + t];
+      ks[c] = *reinterpret_cast<const uint4*>(kb + j * ktok + sub * 16);
+      vs[c] = *reinterpret_cast<const uint4*>(vb + j * vtok + sub * 16);
+    }
+    if (sc)
+      for (int t = threadIdx.x; t < rows; t += kMoveThreads) ss[t] = sc[idx[t0 + t]];
+    __syncthreads();                             // every row of the batch has been read
+    for (int c = threadIdx.x; c < chunks; c += kMoveThreads) {
+      const int t = c / lanes, sub = c % lanes;
+      *reinterpret_cast<uint4*>(kb + (long long)(t0 + t) * ktok + sub * 16) = ks[c];
+      *reinterpret_cast<uint4*>(vb + (long long)(t0 + t) * vtok + sub * 16) = vs[c];
+    }
+    if (sc)
+      for (int t = threadIdx.x; t < rows; t += kMoveThreads) sc[t0 + t] = ss[t];
+    __syncthreads();                             // the staging area is free, and later batches read rows written by none
+  }
+}
+
+}  // namespace
+
+bool step_score_fits(const Plan& pl) {
+  if (pl.r != 1 || pl.G > kStepMaxG || (size_t)pl.G * pl.n * sizeof(float) > kStepMaxLogitBytes) return false;
+  return pl.G <= 8 || pl.G == 12 || pl.G == 16;
+}
+
+ahakv_status launch_step_score(const Plan& pl, const void* q, const void* k, const float* prev, float* score,
+                               cudaStream_t st) {
+  const bool d64 = pl.d == 64;
+  switch (pl.dtype) {
+    case AHAKV_F32: return d64 ? launch_step_g<float, 64>(pl, q, k, prev, score, st) : launch_step_g<float, 128>(pl, q, k, prev, score, st);
+    case AHAKV_F16: return d64 ? launch_step_g<__half, 64>(pl, q, k, prev, score, st) : launch_step_g<__half, 128>(pl, q, k, prev, score, st);
+    default: return d64 ? launch_step_g<__nv_bfloat16, 64>(pl, q, k, prev, score, st)
+                        : launch_step_g<__nv_bfloat16, 128>(pl, q, k, prev, score, st);
+  }
+}
+
+ahakv_status launch_compact_inplace(const Plan& pl, void* k, void* v, float* score, const int32_t* kept_idx,
+                                    cudaStream_t st) {
+  const int row_bytes = pl.d * pl.es;
+  const int per_row = 2 * row_bytes + (int)sizeof(float);
+  int rows_per_batch = kMoveBatchBytes / per_row;
+  rows_per_batch -= rows_per_batch % 4;          // keeps the staged scores 16-byte aligned behind the rows
+  constexpr int kMaxDevices = 64;
+  static bool configured[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AHAKV_ERR_CUDA;
+  if (!configured[dev]) {
+    if (cudaFuncSetAttribute(compact_inplace_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMoveBatchBytes) != cudaSuccess)
+      return AHAKV_ERR_CUDA;
+    configured[dev] = true;
+  }
+  const Shape& shape = pl;
+  compact_inplace_kernel<<<pl.B * pl.Hkv, kMoveThreads, (size_t)rows_per_batch * per_row, st>>>(
+      (char*)k, (char*)v, score, kept_idx, shape, rows_per_batch);
+  count_launch();
+  return cuda_ok(cudaGetLastError());
+}
+
+}  // namespace ahakv

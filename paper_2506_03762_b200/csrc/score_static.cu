@@ -43,15 +43,25 @@ size_t ahakv_static_workspace_bytes(void) { return (size_t)AHAKV_STATIC_WS_BYTES
 
 ahakv_status ahakv_score_static(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
                                 const float* score_prev, float* score, ahakv_stream_t stream) {
-  const size_t need = ahakv_workspace_bytes(p);
-  if (need == 0) return AHAKV_ERR_INVALID_ARG;                    // the parameters themselves are wrong
-  if (need > (size_t)AHAKV_STATIC_WS_BYTES) return AHAKV_ERR_WORKSPACE;   // too large for the built-in scratch
+  ahakv::Plan pl;
+  ahakv_status rc = ahakv::make_plan(p, &pl);                     // the same verdict on the parameters as ahakv_score's
+  if (rc != AHAKV_OK) return rc;
+  if (pl.ws_total > (size_t)AHAKV_STATIC_WS_BYTES) return AHAKV_ERR_WORKSPACE;   // too large for the built-in scratch
   void* ws = nullptr;
-  const ahakv_status rc = static_ws_address(&ws);
+  rc = static_ws_address(&ws);
   if (rc != AHAKV_OK) return rc;
   // Same kernels, same order as ahakv_score; it clears the words of the scratch that must start at
   // zero (and marks the run partials "not published") itself, so what the last call left is harmless.
   return ahakv_score(p, q_obs, k, v, score_prev, score, ws, (size_t)AHAKV_STATIC_WS_BYTES, stream);
+}
+
+// The status word the kernels of the last ahakv_score_static call on this device left at the head of the
+// array: AHAKV_OK, or AHAKV_ERR_TIMEOUT if a bounded device-side wait gave up.  Synchronises `stream`.
+ahakv_status ahakv_static_last_device_status(ahakv_stream_t stream) {
+  void* ws = nullptr;
+  const ahakv_status rc = static_ws_address(&ws);
+  if (rc != AHAKV_OK) return rc;
+  return ahakv_last_device_status(ws, stream);
 }
 
 }  // extern "C"

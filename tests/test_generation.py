@@ -1,0 +1,142 @@
+"""Algorithm 1's generation phase one token at a time on the GPU: the 1 x n score update (``ahakv_score_step``),
+selection, and compaction in place (``ahakv_compact_inplace``), chained for many steps and checked against the
+oracle step by step."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ahakv_oracle as orc
+from paper_2506_03762_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+def _dt(ab, dtype):
+    return {ab.F32: torch.float32, ab.F16: torch.float16, ab.BF16: torch.bfloat16}[dtype]
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,d,n,dtype_name,flags", [
+    (2, 8, 2, 128, 2049, "BF16", 0),           # the shape of a cache held at its budget, grouped queries
+    (1, 4, 4, 128, 700, "F16", 0),
+    (1, 6, 2, 64, 300, "F32", 0),              # three query heads a group, float32 at 1e-5
+    (3, 7, 1, 64, 515, "F16", 4),              # seven heads a group pooled by maximum
+    (1, 1, 1, 128, 1, "F16", 0),               # a single cached token
+])
+def test_score_step_matches_the_oracle_and_the_general_path(B, Hq, Hkv, d, n, dtype_name, flags):
+    from paper_2506_03762_b200 import binding as ab
+    from tests import parity
+    dtype = getattr(ab, dtype_name)
+    g = torch.Generator().manual_seed(n)
+    q = torch.randn((B, Hq, 1, d), generator=g).to(_dt(ab, dtype)).to(DEV)
+    k = torch.randn((B, Hkv, n, d), generator=g).to(_dt(ab, dtype)).to(DEV)
+    prev = (torch.rand((B, Hkv, n), generator=g) * 0.01).to(DEV)
+    p = ab.Params(B, Hq, Hkv, d, n, 1, min(16, n), max(1, n // 2), dtype=dtype, n_total=40000 + n, flags=flags)
+    got = torch.empty((B, Hkv, n), dtype=torch.float32, device=DEV)
+    ab.ahakv_score_step(p, q, k, prev, got)
+    op = parity.oracle_params(p)
+    ref = orc.score(op, synth.to_numpy(q), synth.to_numpy(k), synth.to_numpy(k), prev.double().cpu().numpy())
+    parity.assert_scores_close(p, got.cpu().numpy(), ref, "score_step")
+    general = parity.run_score(p, q, k, k, prev)
+    parity.assert_scores_close(p, got.cpu().numpy(), general.double().cpu().numpy(), "score_step vs ahakv_score")
+    # in place: score_prev and score the same buffer
+    buf = prev.clone()
+    ab.ahakv_score_step(p, q, k, buf, buf)
+    assert torch.equal(buf, got)
+
+
+def test_score_step_declines_what_it_does_not_take():
+    from paper_2506_03762_b200 import binding as ab
+    q = torch.zeros((1, 4, 1, 128), dtype=torch.float16, device=DEV)
+    k = torch.zeros((1, 4, 64, 128), dtype=torch.float16, device=DEV)
+    s = torch.zeros((1, 4, 64), device=DEV)
+    assert ab.ahakv_score_step(ab.Params(1, 4, 4, 128, 64, 1, 4, 8, flags=ab.FLAG_VALUE_PRIOR), q, k, None, s,
+                               check=False) == ab.ERR_UNSUPPORTED
+    assert ab.ahakv_score_step(ab.Params(1, 4, 4, 128, 64, 2, 4, 8, flags=0), q, k, None, s,
+                               check=False) == ab.ERR_INVALID_ARG
+    assert ab.ahakv_score_step(ab.Params(1, 4, 4, 128, 50000, 1, 4, 8, flags=0), 256, 256, None, 256,
+                               check=False) == ab.ERR_UNSUPPORTED          # 50000 logits do not fit in shared memory
+
+
+@pytest.mark.parametrize("dtype_name,d,first_evicted", [("F16", 128, 0), ("BF16", 64, 700), ("F32", 128, 1023), ("F16", 128, None)])
+def test_compact_inplace_equals_the_gather(dtype_name, d, first_evicted):
+    from paper_2506_03762_b200 import binding as ab
+    dtype = getattr(ab, dtype_name)
+    B, H, n, Bud = 2, 3, 1100, 1024
+    g = torch.Generator().manual_seed(d)
+    k = torch.randn((B, H, n, d), generator=g).to(_dt(ab, dtype)).to(DEV)
+    v = torch.randn((B, H, n, d), generator=g).to(_dt(ab, dtype)).to(DEV)
+    s = torch.rand((B, H, n), generator=g).to(DEV)
+    idx = []
+    for u in range(B * H):
+        if first_evicted is None:                                  # nothing among the first Bud rows is evicted
+            keep = torch.arange(Bud)
+        else:
+            tail = first_evicted + torch.randperm(n - first_evicted, generator=g)[: Bud - first_evicted].sort().values
+            keep = torch.cat([torch.arange(first_evicted), tail])
+        idx.append(keep)
+    idx = torch.stack(idx).view(B, H, Bud).to(torch.int32).to(DEV)
+    p = ab.Params(B, H, H, d, n, 8, 16, Bud, dtype=dtype)
+    k_out, v_out, s_out, _ = ab.alloc_outputs(p, DEV)
+    ab.ahakv_compact(p, k, v, s, idx, k_out, v_out, s_out)
+    k2, v2, s2 = k.clone(), v.clone(), s.clone()
+    ab.ahakv_compact_inplace(p, k2, v2, s2, idx)
+    assert torch.equal(k2[:, :, :Bud], k_out) and torch.equal(v2[:, :, :Bud], v_out) and torch.equal(s2[:, :, :Bud], s_out)
+    assert torch.equal(k2[:, :, Bud:], k[:, :, Bud:])              # rows past n_keep are left alone
+    ko, vo, _ = orc.compact(orc.OracleParams(B, H, H, d, n, 8, 16, Bud, dtype=dtype), synth.to_numpy(k),
+                            synth.to_numpy(v), idx.cpu().numpy())
+    assert synth.to_numpy(k2[:, :, :Bud]).tobytes() == ko.tobytes()
+    assert synth.to_numpy(v2[:, :, :Bud]).tobytes() == vo.tobytes()
+    # without the score
+    k3, v3 = k.clone(), v.clone()
+    ab.ahakv_compact_inplace(p, k3, v3, None, idx)
+    assert torch.equal(k3, k2) and torch.equal(v3, v2)
+
+
+def test_evict_every_step_for_64_steps():
+    """The cache is held at its budget: every step appends the new token, updates the score with the one new query
+    per head, keeps the recent window and the best of the rest, and compacts in place (Algorithm 1, Generation).
+    The oracle replays every step from the state the GPU path is in, in double precision: scores within 1e-3, the
+    kept set equal outside the tolerance band, the moved rows byte-exact."""
+    from paper_2506_03762_b200 import binding as ab
+    from tests import parity
+    B, Hq, Hkv, d, Bud, Br, steps, N0 = 2, 8, 2, 128, 256, 16, 64, 5000
+    n = Bud + 1
+    g = torch.Generator().manual_seed(2506)
+    dt = torch.bfloat16
+    k = torch.zeros((B, Hkv, n, d), dtype=dt, device=DEV)
+    v = torch.zeros((B, Hkv, n, d), dtype=dt, device=DEV)
+    k[:, :, :Bud] = torch.randn((B, Hkv, Bud, d), generator=g).to(dt).to(DEV)
+    v[:, :, :Bud] = torch.randn((B, Hkv, Bud, d), generator=g).to(dt).to(DEV)
+    f = torch.zeros((B, Hkv, n), device=DEV)
+    f[:, :, :Bud] = (torch.rand((B, Hkv, Bud), generator=g) * 0.02).to(DEV)
+    idx = torch.empty((B, Hkv, Bud), dtype=torch.int32, device=DEV)
+    evicted_somewhere_other_than_the_end = 0
+    for t in range(steps):
+        p = ab.Params(B, Hq, Hkv, d, n, 1, Br, Bud, dtype=ab.BF16, n_total=N0 + t + 1, flags=0)
+        ws = ab.alloc_workspace(p, DEV)
+        q_t = torch.randn((B, Hq, 1, d), generator=g).to(dt).to(DEV)
+        k[:, :, Bud] = torch.randn((B, Hkv, d), generator=g).to(dt).to(DEV)      # the new token's key and value
+        v[:, :, Bud] = torch.randn((B, Hkv, d), generator=g).to(dt).to(DEV)
+        f[:, :, Bud] = 0.0                                                       # a new token starts at zero
+        k_before, v_before, f_before = k.clone(), v.clone(), f.clone()
+        ab.ahakv_score_step(p, q_t, k, f, f)
+        ab.ahakv_select(p, f, idx, ws)
+        f_scored = f.clone()
+        ab.ahakv_compact_inplace(p, k, v, f, idx)
+        # the oracle, from the same state
+        op = parity.oracle_params(p)
+        ref = orc.evict(op, synth.to_numpy(q_t), synth.to_numpy(k_before), synth.to_numpy(v_before),
+                        f_before.double().cpu().numpy())
+        parity.assert_scores_close(p, f_scored.cpu().numpy(), ref["score"], f"step {t} score")
+        gi = idx.cpu().numpy()
+        for b in range(B):
+            for h in range(Hkv):
+                parity.assert_kept_valid(p, gi[b, h], ref["kept_idx"][b, h], ref["score"][b, h])
+        ko, vo, _ = orc.compact(op, synth.to_numpy(k_before), synth.to_numpy(v_before), gi)
+        assert synth.to_numpy(k[:, :, :Bud]).tobytes() == ko.tobytes(), f"step {t}: K rows"
+        assert synth.to_numpy(v[:, :, :Bud]).tobytes() == vo.tobytes(), f"step {t}: V rows"
+        assert torch.equal(f[:, :, :Bud], torch.gather(f_scored, 2, idx.long()))
+        evicted_somewhere_other_than_the_end += int((gi[..., 0] != 0).sum() + (gi[..., Bud // 2] != Bud // 2).sum())
+    assert evicted_somewhere_other_than_the_end > 0                 # the moves were real ones

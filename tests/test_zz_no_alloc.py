@@ -48,7 +48,7 @@ def test_static_scratch_matches_caller_workspace_twice_in_a_row(name, over):
         want = parity.run_score(p, q, k, v, prev)                       # ahakv_score, caller's workspace
         got = torch.full(shape, float("nan"), dtype=torch.float32, device=dev)
         ab.ahakv_score_static(p, q, k, v, prev, got)
-        torch.cuda.synchronize()
+        assert ab.ahakv_static_last_device_status() == ab.OK        # synchronises the stream
         a, b = got.double().cpu().numpy(), want.double().cpu().numpy()
         assert np.isfinite(a).all()
         assert (np.abs(a - b) <= rtol * np.abs(b) + atol).all()
