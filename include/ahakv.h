@@ -169,6 +169,27 @@ ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k
                          const float* score_prev, void* k_out, void* v_out, float* score_out,
                          int32_t* kept_idx, void* ws, size_t ws_bytes, ahakv_stream_t stream);
 
+/* The whole step for a batch whose sequences differ in length, position and budget (a serving batch).  `p`
+ * describes the allocation: p->n_ctx is the token extent of k, v and score_prev (the longest sequence's room),
+ * p->budget the largest budget; everything else holds for all sequences.  seqs: HOST array of p->batch entries;
+ * sequence b has seqs[b].n_ctx cached rows (obs_window <= n_ctx <= p->n_ctx), has seen seqs[b].n_total tokens and
+ * keeps seqs[b].budget rows (recent_window <= budget <= p->budget).  The heads of one sequence share its budget.
+ * Layouts: q_obs, k, v as described by p (default [B,Hq,r,d] and [B,Hkv,p->n_ctx,d]; rows past a sequence's n_ctx
+ * are not read).  Arrays indexed by token or by kept row are dense per sequence inside the sequence's slot of the
+ * full-size array: score_prev for sequence b starts at b * Hkv * p->n_ctx floats and is [Hkv, n_ctx_b] from there;
+ * k_out, v_out, score_out and kept_idx start at b * Hkv * keep_max rows (keep_max = min(p->n_ctx, p->budget)) and
+ * are [Hkv, min(n_ctx_b, budget_b), ...] from there.  The sequences are queued one after the other on `stream`
+ * with the kernels of ahakv_evict, sharing `ws` (sized for p); each gets exactly what ahakv_evict would give it
+ * alone.  Nothing is queued if any entry is invalid. */
+typedef struct {
+  int32_t n_ctx;
+  int32_t budget;
+  int64_t n_total;
+} ahakv_seq;
+ahakv_status ahakv_evict_ragged(const ahakv_params* p, const ahakv_seq* seqs, const void* q_obs, const void* k,
+                                const void* v, const float* score_prev, void* k_out, void* v_out, float* score_out,
+                                int32_t* kept_idx, void* ws, size_t ws_bytes, ahakv_stream_t stream);
+
 /* Reads the status word the kernels of the last call on this workspace left in `ws` (synchronises
  * `stream`).  AHAKV_OK, or AHAKV_ERR_TIMEOUT if a bounded device-side wait gave up, in which case
  * the call's outputs are not valid. */

@@ -42,6 +42,11 @@ class CParams(ctypes.Structure):
     ]
 
 
+class CSeq(ctypes.Structure):
+    """Mirror of ``ahakv_seq``."""
+    _fields_ = [("n_ctx", ctypes.c_int32), ("budget", ctypes.c_int32), ("n_total", ctypes.c_int64)]
+
+
 @dataclass
 class Params:
     batch: int
@@ -92,6 +97,7 @@ SIGNATURES = {
     "ahakv_select": (ctypes.c_int, [_PP, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_compact": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_evict": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_evict_ragged": (ctypes.c_int, [_PP, ctypes.POINTER(CSeq), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_score_static": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_static_workspace_bytes": (_sz, []),
     "ahakv_static_last_device_status": (ctypes.c_int, [_vp]),
@@ -270,6 +276,19 @@ def ahakv_evict(p: Params, q_obs, k, v, score_prev, k_out, v_out, score_out, kep
                            _ptr(v_out), _ptr(score_out), _ptr(kept_idx), _ptr(ws), nbytes, _stream(stream))
     if check:
         _raise(st, "ahakv_evict")
+    return st
+
+
+def ahakv_evict_ragged(p: Params, seqs, q_obs, k, v, score_prev, k_out, v_out, score_out, kept_idx, ws,
+                       ws_bytes: int | None = None, stream=None, check: bool = True) -> int:
+    """``seqs``: one (n_ctx, budget, n_total) triple per sequence."""
+    cp = p.c()
+    arr = (CSeq * len(seqs))(*[CSeq(int(a), int(b), int(c)) for a, b, c in seqs])
+    nbytes = ws.numel() * ws.element_size() if ws_bytes is None else ws_bytes
+    st = lib().ahakv_evict_ragged(ctypes.byref(cp), arr, _ptr(q_obs), _ptr(k), _ptr(v), _ptr(score_prev), _ptr(k_out),
+                                  _ptr(v_out), _ptr(score_out), _ptr(kept_idx), _ptr(ws), nbytes, _stream(stream))
+    if check:
+        _raise(st, "ahakv_evict_ragged")
     return st
 
 

@@ -362,6 +362,41 @@ ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k
   return rc;
 }
 
+ahakv_status ahakv_evict_ragged(const ahakv_params* p, const ahakv_seq* seqs, const void* q_obs, const void* k,
+                                const void* v, const float* score_prev, void* k_out, void* v_out, float* score_out,
+                                int32_t* kept_idx, void* ws, size_t ws_bytes, ahakv_stream_t stream) {
+  Plan outer;
+  ahakv_status rc = make_plan(p, &outer);        // p describes the allocation: n_ctx and budget are the largest of the batch
+  if (rc) return rc;
+  if (!seqs) return AHAKV_ERR_INVALID_ARG;
+  if ((rc = check_ws(outer, ws, ws_bytes))) return rc;
+  // every sequence is checked before anything is queued
+  for (int b = 0; b < outer.B; ++b) {
+    if (seqs[b].n_ctx < outer.r || seqs[b].n_ctx > p->n_ctx || seqs[b].budget < 1 || seqs[b].budget > p->budget ||
+        seqs[b].budget < p->recent_window || seqs[b].n_total < seqs[b].n_ctx)
+      return AHAKV_ERR_INVALID_ARG;
+  }
+  const size_t es = outer.es, keep_max = outer.n_keep;
+  const size_t row = (size_t)outer.d * es;
+  for (int b = 0; b < outer.B; ++b) {
+    ahakv_params pb = *p;
+    pb.batch = 1;
+    pb.n_ctx = seqs[b].n_ctx;
+    pb.n_total = seqs[b].n_total;
+    pb.budget = seqs[b].budget;
+    for (int t = 0; t < 3; ++t) { pb.q_stride[t] = outer.qs[t]; pb.k_stride[t] = outer.ks[t]; pb.v_stride[t] = outer.vs[t]; }
+    const char* qb = (const char*)q_obs + (size_t)b * outer.qs[0] * es;
+    const char* kb = (const char*)k + (size_t)b * outer.ks[0] * es;
+    const char* vb = (const char*)v + (size_t)b * outer.vs[0] * es;
+    const size_t tok = (size_t)b * outer.Hkv * outer.n, kept = (size_t)b * outer.Hkv * keep_max;
+    rc = ahakv_evict(&pb, qb, kb, vb, score_prev ? score_prev + tok : nullptr, (char*)k_out + kept * row,
+                     (char*)v_out + kept * row, score_out ? score_out + kept : nullptr, kept_idx + kept, ws, ws_bytes,
+                     stream);
+    if (rc) return rc;
+  }
+  return AHAKV_OK;
+}
+
 ahakv_status ahakv_last_device_status(const void* ws, ahakv_stream_t stream) {
   if (!ws) return AHAKV_ERR_WORKSPACE;
   int word = 0;
