@@ -237,6 +237,17 @@ ahakv_status ahakv_static_last_device_status(ahakv_stream_t stream);
 ahakv_status ahakv_score_static(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
                                 const float* score_prev, float* score, ahakv_stream_t stream);
 
+/* For tests of the failure path only (no counterpart in the paper).  Every wait inside the tensor-core scoring
+ * kernel on something another thread, the copy engine, the tensor core or another CTA must deliver is bounded
+ * (1 s); when one runs out the kernel records AHAKV_ERR_TIMEOUT in the workspace's status word and winds down
+ * without trapping, so the context stays usable.  wait_ms > 0 shortens that limit for the launches that follow
+ * (0 restores 1 s); withhold_first_partial != 0 plants the fault that makes a wait run out: the softmax
+ * statistics of the first run of the first row block are never published, so whoever merges that row block waits
+ * in vain.  While either is set, launches use a second instantiation of the same kernel code that takes the limit
+ * and the fault from its arguments; the instantiation every other call runs has neither.  Process-wide; not for
+ * production use. */
+void ahakv_test_set_wait(int32_t wait_ms, int32_t withhold_first_partial);
+
 /* Number of kernels the library has launched in this process since it was loaded. */
 int64_t ahakv_launch_count(void);
 

@@ -102,6 +102,7 @@ SIGNATURES = {
     "ahakv_static_workspace_bytes": (_sz, []),
     "ahakv_static_last_device_status": (ctypes.c_int, [_vp]),
     "ahakv_last_device_status": (ctypes.c_int, [_vp, _vp]),
+    "ahakv_test_set_wait": (None, [ctypes.c_int32, ctypes.c_int32]),
     "ahakv_launch_count": (ctypes.c_int64, []),
     "ahakv_profile_enable": (ctypes.c_int, [ctypes.c_int]),
     "ahakv_profile_read": (ctypes.c_int64, [ctypes.POINTER(ctypes.c_double)]),
@@ -158,6 +159,10 @@ def ahakv_workspace_bytes(p: Params) -> int:
 
 def ahakv_lambda(n_total: int, budget: int, head_dim: int) -> float:
     return float(lib().ahakv_lambda(n_total, budget, head_dim))
+
+
+def ahakv_test_set_wait(wait_ms: int, withhold_first_partial: bool) -> None:
+    lib().ahakv_test_set_wait(int(wait_ms), 1 if withhold_first_partial else 0)
 
 
 def ahakv_launch_count() -> int:

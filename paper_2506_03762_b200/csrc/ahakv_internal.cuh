@@ -56,6 +56,7 @@ ahakv_status launch_score_simt(const Plan& pl, const void* q, const void* k, flo
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
                              float2* partial, int* counters, int* status, cudaStream_t st);
 bool score_tc_available();
+void score_tc_test_hooks(long long wait_ns, int withhold);   // see ahakv_test_set_wait
 // The generation phase one token at a time (decode.cu): the score update of one new query per head without
 // scratch memory, and compaction in place.
 bool step_score_fits(const Plan& pl);

@@ -406,6 +406,10 @@ ahakv_status ahakv_last_device_status(const void* ws, ahakv_stream_t stream) {
   return word == 0 ? AHAKV_OK : AHAKV_ERR_TIMEOUT;
 }
 
+void ahakv_test_set_wait(int32_t wait_ms, int32_t withhold_first_partial) {
+  score_tc_test_hooks((long long)wait_ms * 1000000LL, withhold_first_partial != 0);
+}
+
 int64_t ahakv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* ahakv_status_string(ahakv_status s) {

@@ -57,6 +57,8 @@
 // and winds down.
 #include <cuda.h>
 
+#include <atomic>
+
 #include "ahakv_internal.cuh"
 #include "tc_common.cuh"
 
@@ -94,7 +96,16 @@ struct TcArgs {
   float* nu;         // [B * Hkv][n]
   int* ctr;          // [2] next pass-1 run, next pass-2 run (zero at launch)
   int* status;
+  long long test_wait_ns;   // test build of the kernel only: what every bounded wait allows
+  int test_withhold;        // test build only: the partial of the first run of the first row block is never published
 };
+
+// The kernel exists twice: the one every call runs, whose waits allow kWaitLimitNs, and a second instantiation that
+// takes the limit and a planted fault from its arguments, for the test of the failure path (ahakv_test_set_wait).
+// Same code, same wind-down; only these two lines differ.
+template <bool kTest> __device__ __forceinline__ long long wait_limit(const TcArgs& a) {
+  return kTest ? a.test_wait_ns : kWaitLimitNs;
+}
 
 // ---- shared memory layout --------------------------------------------------------------------
 struct __align__(8) Barriers {
@@ -178,7 +189,9 @@ __device__ __forceinline__ int seg_peek(Shared* sh, int idx) {
   return ld_volatile(&sh->seg[idx % kSegRing]);
 }
 // The same, waiting (bounded) for the scheduler.  kSegEnd ends the sequence; so does a wait that ran out.
-__device__ __forceinline__ int seg_get(Shared* sh, int idx, int* status) {
+// Readers allow twice the time the scheduler's own thread does: when nothing moves, that thread gives up first and
+// publishes kSegEnd, so every reader of the CTA sees the same end of the sequence rather than its own.
+__device__ __forceinline__ int seg_get(Shared* sh, int idx, int* status, long long limit_ns) {
   int e = seg_peek(sh, idx);
   if (e != -2) return e;
   long long t0 = -1;
@@ -187,13 +200,13 @@ __device__ __forceinline__ int seg_get(Shared* sh, int idx, int* status) {
     if ((e = seg_peek(sh, idx)) != -2) return e;
     if ((spins & 255) != 255) continue;                   // the clock is slow to read
     if (t0 < 0) t0 = now_ns();
-    else if (now_ns() - t0 > kWaitLimitNs) {
+    else if (now_ns() - t0 > 2 * limit_ns) {
       atomicExch(status, (int)AHAKV_ERR_TIMEOUT);
       return kSegEnd;
     }
   }
 }
-__device__ __forceinline__ int mrg_get(Shared* sh, int idx, int* status) {
+__device__ __forceinline__ int mrg_get(Shared* sh, int idx, int* status, long long limit_ns) {
   const long long t0 = now_ns();
   for (;;) {
     if (idx < ld_volatile(&sh->mrg_pub)) {
@@ -201,7 +214,7 @@ __device__ __forceinline__ int mrg_get(Shared* sh, int idx, int* status) {
       return ld_volatile(&sh->mrg[idx % kMergeRing]);
     }
     __nanosleep(200);
-    if (now_ns() - t0 > kWaitLimitNs) {
+    if (now_ns() - t0 > 2 * limit_ns) {
       atomicExch(status, (int)AHAKV_ERR_TIMEOUT);
       return kSegEnd;
     }
@@ -209,10 +222,10 @@ __device__ __forceinline__ int mrg_get(Shared* sh, int idx, int* status) {
 }
 
 // f(pass, run) for every segment of this CTA, in order.
-template <typename F>
+template <bool kTest, typename F>
 __device__ __forceinline__ void for_each_segment(const TcArgs& a, Shared* sh, F f) {
   for (int idx = 0;; ++idx) {
-    const int e = seg_get(sh, idx, a.status);
+    const int e = seg_get(sh, idx, a.status, wait_limit<kTest>(a));
     if (e == kSegEnd) return;
     f(e & 1, e >> 1, idx);
   }
@@ -276,10 +289,11 @@ struct VCursor {
 };
 // Moves to the first stage of the next segment that brings value rows.  1: found, 0: the sequence has ended,
 // -1: not published yet (only when `block` is false).
+template <bool kTest>
 __device__ __forceinline__ int v_seek(const TcArgs& a, Shared* sh, VCursor& c, bool block, int* behind = nullptr) {
   for (;; ++c.idx) {
     if (behind) *(volatile int*)behind = c.idx;               // everything before c.idx has been dealt with
-    const int e = block ? seg_get(sh, c.idx, a.status) : seg_peek(sh, c.idx);
+    const int e = block ? seg_get(sh, c.idx, a.status, wait_limit<kTest>(a)) : seg_peek(sh, c.idx);
     if (e == -2) return -1;
     if (e == kSegEnd) return 0;
     if (e & 1) continue;
@@ -295,6 +309,7 @@ __device__ __forceinline__ int v_seek(const TcArgs& a, Shared* sh, VCursor& c, b
 // TMA producer: one thread keeps the CTA's sequence of segments filled (scheduler rounds) and feeds two
 // independent streams, whichever has a free slot: Q and K tiles in the order of the sequence, and the value
 // rows that go with the pass-1 key tiles.
+template <bool kTest>
 __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtensorMap* kmap, const CUtensorMap* vmap,
                          Shared* sh, char* tiles) {
   Barriers* bars = &sh->bars;
@@ -361,7 +376,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
       }
     }
     if (v_state == 0) {
-      const int f = v_seek(a, sh, vcur, false);
+      const int f = v_seek<kTest>(a, sh, vcur, false);
       if (f == 1) { v_state = 2; progress = true; }
       else if (f == 0) { v_state = 3; progress = true; }
     }
@@ -383,7 +398,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
     } else if ((++idle_spins & 1023) == 0) {               // the clock is slow to read: look at it rarely
       const long long now = now_ns();
       if (idle_since < 0) idle_since = now;
-      else if (now - idle_since > kWaitLimitNs) {
+      else if (now - idle_since > wait_limit<kTest>(a)) {
         atomicExch(a.status, (int)AHAKV_ERR_TIMEOUT);
         if (!sched.done) { sched_announce(sh, sched, kSegEnd); sched_publish(sh, sched, kSegEnd); }
         // wind down: give copies already in flight a bounded time (1 ms) to land before the CTA exits
@@ -397,6 +412,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
 // Value-norm group (four warps, 128 threads): two adjacent lanes share a row of each 64-row stage of the
 // V ring (one half of its 16-byte chunks each, in an order that keeps them on different banks), square
 // and add in FP32 and meet by shuffle: nu_j = |V_j|^2.
+template <bool kTest>
 __device__ void v_group(const TcArgs& a, Shared* sh, char* tiles) {
   Barriers* bars = &sh->bars;
   const int row = (threadIdx.x & 127) >> 1, sub = threadIdx.x & 1;
@@ -404,10 +420,10 @@ __device__ void v_group(const TcArgs& a, Shared* sh, char* tiles) {
   VCursor cc;
   cc.idx = 0;
   int ci = 0;
-  while (v_seek(a, sh, cc, true, leader ? &sh->seg_done_v : nullptr) == 1) {
+  while (v_seek<kTest>(a, sh, cc, true, leader ? &sh->seg_done_v : nullptr) == 1) {
     for (; cc.t < cc.cnt; ++cc.t, ++ci) {
       const int vs = ci % kVStages;
-      if (!mbar_wait(&bars->v_full[vs], (ci / kVStages) & 1, a.status)) return;
+      if (!mbar_wait(&bars->v_full[vs], (ci / kVStages) & 1, a.status, wait_limit<kTest>(a))) return;
       const char* stage = tiles + kOffV + vs * kVStageBytes;
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -438,23 +454,24 @@ __device__ void v_group(const TcArgs& a, Shared* sh, char* tiles) {
 
 // MMA issuer (one thread).
 // Pass 1: D[rows x keys] = Q K^T.  Pass 2: D[keys x rows] = K Q^T - off / c.
+template <bool kTest>
 __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tmem_base) {
   Barriers* bars = &sh->bars;
   int tc = 0, sc = 0, pc = 0;
   bool ok = true;
   const uint64_t fold_desc = umma_desc_ext(smem_u32(tiles + kOffExt + 2 * kExtBytes));
   const int nk = a.D / 16;
-  for_each_segment(a, sh, [&](int pass, int run, int) {
+  for_each_segment<kTest>(a, sh, [&](int pass, int run, int) {
     if (!ok) return;
     const Run rn = run_info(a, run);
     const int qb = sc & 1;
-    if (!(ok = mbar_wait(&bars->q_full[qb], (sc >> 1) & 1, a.status))) return;
+    if (!(ok = mbar_wait(&bars->q_full[qb], (sc >> 1) & 1, a.status, wait_limit<kTest>(a)))) return;
     uint32_t idesc = umma_idesc(128, 128, a.bf16);
     uint64_t ext_desc = 0;
     const int slot = pc & 1;
     if (pass == 1) {
       // the row block's offset extension, from this CTA's merge group
-      if (!(ok = mbar_wait(&bars->ext_full[slot], (pc >> 1) & 1, a.status))) return;
+      if (!(ok = mbar_wait(&bars->ext_full[slot], (pc >> 1) & 1, a.status, wait_limit<kTest>(a)))) return;
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       idesc = umma_idesc(128, unit_info(a, rn.unit).npad, a.bf16);
       ext_desc = umma_desc_ext(smem_u32(tiles + kOffExt + slot * kExtBytes));
@@ -462,8 +479,8 @@ __device__ void mma_issuer(const TcArgs& a, Shared* sh, char* tiles, uint32_t tm
     for (int t = 0; t < rn.cnt; ++t, ++tc) {
       const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
       const int acc = tc & 3, aph = (tc >> 2) & 1;      // the four accumulators in turn
-      if (!(ok = mbar_wait(&bars->acc_empty[acc], aph ^ 1, a.status))) return;
-      if (!(ok = mbar_wait(&bars->k_full[stage], ph, a.status))) return;
+      if (!(ok = mbar_wait(&bars->acc_empty[acc], aph ^ 1, a.status, wait_limit<kTest>(a)))) return;
+      if (!(ok = mbar_wait(&bars->k_full[stage], ph, a.status, wait_limit<kTest>(a)))) return;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + (uint32_t)(acc * 128);
       const uint32_t q_lo = umma_desc_lo(smem_u32(tiles + kOffQ + qb * kQBytes));
@@ -592,13 +609,14 @@ __device__ __forceinline__ float column_sum_fast(const TcArgs& a, uint32_t taddr
 //           partial, log2 of the sum, with one 4-byte store.
 //   pass 2: thread `jl` owns key j0 + jl over its quarter of the stacked rows; three groups hand their partial
 //           sums over through shared memory, the first adds the four in a fixed order and stores.
+template <bool kTest>
 __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint32_t tmem_base, int g) {
   Barriers* bars = &sh->bars;
   const int s = threadIdx.x & 127, quarter = (threadIdx.x >> 5) & 3;
   const uint32_t lane_base = tmem_base + ((uint32_t)(quarter * 32) << 16);
   int tc = 0, p1c = 0;   // tiles and pass-1 runs seen so far
   bool gone = false;   // a wait ran out: keep only the barriers
-  for_each_segment(a, sh, [&](int pass, int run, int idx) {
+  for_each_segment<kTest>(a, sh, [&](int pass, int run, int idx) {
     const Run rn = run_info(a, run);
     const UnitInfo u = unit_info(a, rn.unit);
     if (pass == 0) {
@@ -609,7 +627,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
       for (int t = 0; t < rn.cnt; ++t, ++tc) {
         if (gone) continue;
         const int acc = tc & 3, aph = (tc >> 2) & 1;
-        if (!mbar_wait(&bars->acc_full[acc], aph, a.status)) { gone = true; continue; }
+        if (!mbar_wait(&bars->acc_full[acc], aph, a.status, wait_limit<kTest>(a))) { gone = true; continue; }
         tc_fence_after();
         const int j0 = (rn.blk0 + t) * kKeyTile + 32 * g;
         const bool full = (rn.blk0 + t) * kKeyTile + kKeyTile - 1 <= a.min_last;   // no key of the tile is masked
@@ -638,7 +656,8 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
         }
         float L = z > 0.f ? m + log2f(z) : -INFINITY;
         if (L != L) L = INFINITY;                            // NaN inputs: never publish the 'not yet' pattern
-        st_partial(&a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s], L);
+        if (!(kTest && a.test_withhold && rn.unit == 0 && rn.rin == 0))
+          st_partial(&a.partial[((size_t)rn.unit * a.rpu + rn.rin) * 128 + s], L);
       }
     } else {
       const int jl = s;
@@ -651,7 +670,7 @@ __device__ __forceinline__ void softmax_group(const TcArgs& a, Shared* sh, uint3
         const int buf = tc & 1, acc = tc & 3, aph = (tc >> 2) & 1;
         const int j0 = (rn.blk0 + t) * kKeyTile, j = j0 + jl;
         float sum = 0.f;
-        if (!gone && !mbar_wait(&bars->acc_full[acc], aph, a.status)) gone = true;
+        if (!gone && !mbar_wait(&bars->acc_full[acc], aph, a.status, wait_limit<kTest>(a))) gone = true;
         if (!gone) {
           tc_fence_after();
           const bool full = j0 + kKeyTile - 1 <= a.min_last;
@@ -724,15 +743,16 @@ __device__ __forceinline__ void write_extension(char* ext, int row, float off, f
 // ahead of the MMA warp: thread `s` waits until the partials of rows 2s and 2s + 1 have arrived from all runs of the
 // row block, merges them in run order into the rows' offsets and writes their offset extensions into
 // shared memory.
+template <bool kTest>
 __device__ void merge_group(const TcArgs& a, Shared* sh, char* tiles, int s) {
   Barriers* bars = &sh->bars;
   for (int mc = 0;; ++mc) {
-    const int run = mrg_get(sh, mc, a.status);
+    const int run = mrg_get(sh, mc, a.status, wait_limit<kTest>(a));
     if (run == kSegEnd) return;
     const Run rn = run_info(a, run);
     const UnitInfo u = unit_info(a, rn.unit);
     const int slot = mc & 1;
-    if (!mbar_wait(&bars->ext_empty[slot], ((mc >> 1) & 1) ^ 1, a.status)) return;
+    if (!mbar_wait(&bars->ext_empty[slot], ((mc >> 1) & 1) ^ 1, a.status, wait_limit<kTest>(a))) return;
     const float2* p = reinterpret_cast<const float2*>(a.partial + (size_t)rn.unit * a.rpu * 128) + s;
     float M0 = -INFINITY, Z0 = 0.f, M1 = -INFINITY, Z1 = 0.f;   // running shift and sum of 2^{L - shift}, per row
     for (int t0 = 0; t0 < a.rpu; t0 += 16) {              // 16 8-byte loads in flight per thread
@@ -753,7 +773,7 @@ __device__ void merge_group(const TcArgs& a, Shared* sh, char* tiles, int s) {
           __nanosleep(400);
           const float2 x = ld_partial2(&p[(size_t)(t0 + missing) * 64]);
           if (x.x == x.x && x.y == x.y) break;
-          if (now_ns() - tstart > kWaitLimitNs) { timed_out = true; break; }
+          if (now_ns() - tstart > wait_limit<kTest>(a)) { timed_out = true; break; }
         }
         if (timed_out) {
           // nothing more is delivered; the MMA warp's own wait then runs out too
@@ -788,6 +808,7 @@ __device__ void merge_group(const TcArgs& a, Shared* sh, char* tiles, int s) {
   }
 }
 
+template <bool kTest>
 __global__ void __launch_bounds__(kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
                 const __grid_constant__ CUtensorMap vmap, const __grid_constant__ TcArgs a) {
@@ -857,15 +878,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
   const uint32_t tmem_base = sh->tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) producer(a, &qmap, &kmap, &vmap, sh, tiles);
+    if (lane == 0) producer<kTest>(a, &qmap, &kmap, &vmap, sh, tiles);
   } else if (warp == 1) {
-    if (lane == 0) mma_issuer(a, sh, tiles, tmem_base);
+    if (lane == 0) mma_issuer<kTest>(a, sh, tiles, tmem_base);
   } else if (warp < 4) {
-    merge_group(a, sh, tiles, threadIdx.x & 63);
+    merge_group<kTest>(a, sh, tiles, threadIdx.x & 63);
   } else if (warp < 20) {
-    softmax_group(a, sh, tmem_base, (warp - 4) >> 2);
+    softmax_group<kTest>(a, sh, tmem_base, (warp - 4) >> 2);
   } else {
-    if (a.prior) v_group(a, sh, tiles);
+    if (a.prior) v_group<kTest>(a, sh, tiles);
   }
 
   tc_fence_before();
@@ -882,6 +903,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap qmap, const __grid_constant_
 
 bool score_tc_available() { return encode_fn() != nullptr; }
 
+// Test hooks (see ahakv_test_set_wait): the limit of the kernel's bounded waits, and a planted fault.  While either
+// is set, launches go to the test instantiation of the kernel.
+static std::atomic<long long> g_test_wait_ns{0};
+static std::atomic<int> g_test_withhold{0};
+void score_tc_test_hooks(long long wait_ns, int withhold) {
+  g_test_wait_ns.store(wait_ns > 0 ? wait_ns : 0);
+  g_test_withhold.store(withhold);
+}
+
 ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const void* v, float* s_raw, float* nu,
                              float2* partial_ws, int* counters, int* status, cudaStream_t st) {
   // once per device: its SM count, and leave to use more than 48 KB of dynamic shared memory
@@ -892,7 +922,8 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   if (sm_count[dev] == 0) {
     int count = 0;
     if (cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || count <= 0 ||
-        cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        cudaFuncSetAttribute(score_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(score_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
       return AHAKV_ERR_CUDA;
     sm_count[dev] = count;
   }
@@ -919,6 +950,10 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   a.partial = reinterpret_cast<float*>(partial_ws); a.s_raw = s_raw; a.nu = nu;
   a.ctr = counters;
   a.status = status;
+  a.test_wait_ns = g_test_wait_ns.load();
+  a.test_withhold = g_test_withhold.load();
+  const bool test = a.test_wait_ns > 0 || a.test_withhold != 0;
+  if (a.test_wait_ns <= 0) a.test_wait_ns = kWaitLimitNs;
 
   CUtensorMap qmap, kmap, vmap;
   const int q_box_rows = pl.r <= 128 ? pl.r : 128, q_box_heads = pl.r <= 128 ? pl.heads_per_rb : 1;
@@ -934,8 +969,8 @@ ahakv_status launch_score_tc(const Plan& pl, const void* q, const void* k, const
   // every partial starts as NaN: "not published yet"
   if (cudaMemsetAsync(a.partial, 0xff, (size_t)a.n_runs * 128 * sizeof(float), st) != cudaSuccess) return AHAKV_ERR_CUDA;
   void* args[] = {&qmap, &kmap, &vmap, &a};
-  const cudaError_t e = cudaLaunchCooperativeKernel((const void*)score_tc_kernel, dim3(grid), dim3(kThreads), args,
-                                                    (size_t)kSmemBytes, st);
+  const void* kernel = test ? (const void*)score_tc_kernel<true> : (const void*)score_tc_kernel<false>;
+  const cudaError_t e = cudaLaunchCooperativeKernel(kernel, dim3(grid), dim3(kThreads), args, (size_t)kSmemBytes, st);
   count_launch();
   if (e != cudaSuccess) return AHAKV_ERR_CUDA;
   return cuda_ok(cudaGetLastError());

@@ -53,7 +53,7 @@ __device__ __forceinline__ bool mbar_test(void* bar, int parity) {
 // Bounded wait.  Returns false (and records the timeout) if the phase did not complete in time.  The
 // clock is slow to read, so it is looked at only after many failed tries (each of which already sleeps in
 // hardware for a while).
-__device__ __forceinline__ bool mbar_wait(void* bar, int parity, int* status) {
+__device__ __forceinline__ bool mbar_wait(void* bar, int parity, int* status, long long limit_ns = kWaitLimitNs) {
 #pragma unroll 1
   for (int t = 0; t < 256; ++t)
     if (mbar_try(bar, parity)) return true;
@@ -62,7 +62,7 @@ __device__ __forceinline__ bool mbar_wait(void* bar, int parity, int* status) {
 #pragma unroll 1
     for (int t = 0; t < 256; ++t)
       if (mbar_try(bar, parity)) return true;
-    if (now_ns() - t0 > kWaitLimitNs) {
+    if (now_ns() - t0 > limit_ns) {
       atomicExch(status, (int)AHAKV_ERR_TIMEOUT);
       return false;
     }
