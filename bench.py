@@ -30,10 +30,15 @@ def parse_args():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=32)
     ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--repeats", type=int, default=10,
+                    help="the block of --steps calls is timed this many times; ms_per_step is the median block")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--resident-layers", type=int, default=4,
-                    help="distinct layers of input kept in HBM and cycled through")
+                    help="distinct layers of input kept in HBM and cycled through (at least; more when one "
+                         "layer's K and V are small against L2)")
+    ap.add_argument("--no-protocol", action="store_true",
+                    help="decode_round only: skip the 256-step protocol (8 chained rounds, evict-every-step)")
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling small cases)")
@@ -64,6 +69,33 @@ def algorithmic_work(w):
     per_token = 4 * w.batch * w.n_kv_heads * w.n_ctx
     score_bytes = kv_read // 2 + q_read + per_token + ((kv_read // 2 + per_token) if w.value_prior else 0)
     return dict(bytes=kv_read + q_read + kv_write, flops=flops, score_bytes=score_bytes)
+
+
+L2_BYTES = 126e6
+
+
+def kernel_source_digest():
+    """sha1 of the scoring kernel's sources: DRAM counters taken from an older kernel are not reported."""
+    import hashlib
+    h = hashlib.sha1()
+    for name in ("score_tc.cu", "tc_common.cuh"):
+        with open(os.path.join(ROOT, "paper_2506_03762_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def measured_traffic(w):
+    """DRAM bytes of one launch of the scoring kernel from the tracked ncu summary (profiles/*.json): counters of a
+    small case (batch 2), scaled by the units a launch of this run processes -- traffic grows with them.  None when
+    there is no summary for this workload or the kernel has changed since the counters were taken."""
+    path = os.path.join(ROOT, "profiles", f"score_tc_kernel_{w.name}.json")
+    if not os.path.exists(path):
+        return None, None
+    d = json.load(open(path))
+    if d.get("kernel_source_sha1") != kernel_source_digest() or bool(d.get("value_prior")) != bool(w.value_prior):
+        return None, os.path.relpath(path, ROOT) + " (stale: the kernel has changed since)"
+    per_unit = (d["dram_bytes_read"] + d["dram_bytes_write"]) / float(d["units"])
+    return per_unit * w.batch * w.n_kv_heads, os.path.relpath(path, ROOT)
 
 
 class ClockSampler:
@@ -192,14 +224,29 @@ def run_reference(args):
     }))
 
 
-def workload_config(w, args):
+def kv_bytes(w):
+    return 2 * w.batch * w.n_kv_heads * w.n_ctx * w.head_dim * w.elem_size
+
+
+def resident_copies(w, args):
+    """Distinct seeded layers kept in HBM: enough that a step never finds its inputs in L2 (the copies between
+    two uses of a layer amount to at least twice L2), within 48 GB."""
+    need = int(-(-2 * L2_BYTES // kv_bytes(w))) + 1
+    cap = max(1, int(48e9 // max(kv_bytes(w), 1)))
+    return max(1, min(max(args.resident_layers, need), cap))
+
+
+def workload_config(w, args, copies=None):
+    copies = resident_copies(w, args) if copies is None else copies
     return {"workload": w.name, "batch": w.batch, "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads,
             "head_dim": w.head_dim, "n_ctx": w.n_ctx, "obs_window": w.obs_window,
             "recent_window": w.recent_window, "budget": w.budget, "layers_per_pass": w.n_layers,
-            "resident_layers": args.resident_layers, "value_prior": w.value_prior,
+            "resident_layers": copies, "value_prior": w.value_prior,
             "scale_mode": "adaptive_row", "pool_kernel": w.pool_kernel,
-            "l2": "each step's inputs (K+V of a layer) are larger than L2 and steps cycle through "
-                  "distinct resident layers", "parallelism": "replicas only"}
+            "l2": f"steps cycle through {copies} distinct seeded layers resident in HBM, "
+                  f"{copies * kv_bytes(w) / 1e6:.0f} MB of K and V against {L2_BYTES / 1e6:.0f} MB of L2, so no step finds "
+                  "its inputs in L2; warm_ms_per_step is the same call repeated on one layer",
+            "parallelism": "replicas only"}
 
 
 def run_ours(args):
@@ -226,7 +273,7 @@ def run_ours(args):
     p = ab.Params(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.n_ctx, w.obs_window, w.recent_window,
                   w.budget, dtype={"f32": ab.F32, "f16": ab.F16, "bf16": ab.BF16}[w.dtype],
                   n_total=w.n_total, pool_kernel=w.pool_kernel, flags=flags)
-    L = max(1, min(args.resident_layers, max(w.n_layers, 1)))
+    L = resident_copies(w, args)
     layers = [synth.make_layer(w, layer=l, device=dev, seed=synth.BASE_SEED + rank) for l in range(L)]
     prev = synth.make_score_prev(w, device=dev, new_rows=w.obs_window) if w.n_total is not None else None
     ws = ab.alloc_workspace(p, dev)
@@ -255,22 +302,36 @@ def run_ours(args):
         return
     assert ab.ahakv_last_device_status(ws) == ab.OK, "device-side wait timed out during warm-up"
 
-    # ---- timed region: exactly K steps, device-timed -------------------------------------------------
+    # ---- timed region: blocks of exactly K steps, each bracketed and device-timed; the median block counts ------
     sampler = ClockSampler(local) if rank == 0 else None
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = ab.ahakv_launch_count()
-    barrier()
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
-    barrier()
-    ms_total = e0.elapsed_time(e1)
-    launches = ab.ahakv_launch_count() - launches0
+    blocks = []
+    launches = 0
+    for rep in range(max(1, args.repeats)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches0 = ab.ahakv_launch_count()
+        barrier()
+        e0.record(stream)
+        for i in range(args.steps):
+            step(rep * args.steps + i)
+        e1.record(stream)
+        barrier()
+        launches = ab.ahakv_launch_count() - launches0
+        blocks.append(max_over_ranks(e0.elapsed_time(e1), world, dev))
     clocks = sampler.stop() if sampler else None
     status = ab.ahakv_last_device_status(ws)
-    ms_total = max_over_ranks(ms_total, world, dev)
+    ms_total = statistics.median(blocks)
     ms_step = ms_total / args.steps
+    # the same call repeated on one resident layer (inputs that fit in L2 stay there)
+    w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        step(0)
+    barrier()
+    w0.record(stream)
+    for _ in range(args.steps):
+        step(0)
+    w1.record(stream)
+    barrier()
+    warm_ms_step = max_over_ranks(w0.elapsed_time(w1), world, dev) / args.steps
     tokens_per_step = w.batch * w.n_ctx
     value = whole_job_value(tokens_per_step, world, ms_step)
 
@@ -329,20 +390,21 @@ def run_ours(args):
                    "compact": 2 * 2 * w.batch * w.n_kv_heads * w.n_keep * w.head_dim * w.elem_size}
     dom = "score"
     achieved = stage_bytes[dom] / (stage_ms[dom] * 1e-3) / 1e9 if stage_ms[dom] > 0 else 0.0
-    # DRAM bytes of one launch from the ncu capture summarised in profiles/score_tc_kernel_long32k_b2.txt:
-    # 1108.4 MB at batch 2, scaled by the units a launch of this run processes (traffic grows with them).
-    traffic = None
-    if w.name == "long_32k" and w.value_prior:
-        traffic = 1108.4e6 * w.batch / 2
-    roofline = {"kernel": "score_tc_kernel (logits, SG-softmax, column sums, value norms)", "bound": "hbm",
-                "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": achieved / pk["hbm_gbs"],
-                "peak_source": f"{pk['source']} (sustained copy)", "traffic": traffic,
+    traffic, traffic_source = measured_traffic(w)
+    roofline = {"kernel": "score_tc_kernel (logits, SG-softmax, column sums, value norms): the dominant kernel alone; "
+                          "the whole step against its roofline is path_roofline",
+                "bound": "hbm", "achieved": achieved, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / pk["hbm_gbs"], "peak_source": f"{pk['source']} (sustained copy)",
+                "traffic": traffic, "traffic_source": traffic_source,
                 "algorithmic_bytes_per_launch": stage_bytes[dom], "ms_per_launch": stage_ms[dom],
                 "slowest_stage": top}
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": n_warm, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": workload_config(w, args),
+        "vs_baseline": None, "dtype": w.dtype, "data": "synthetic", "config": workload_config(w, args, L),
+        "repeats": len(blocks), "ms_per_step_min": min(blocks) / args.steps,
+        "ms_per_step_max": max(blocks) / args.steps, "block_ms_per_step": [b_ / args.steps for b_ in blocks],
+        "warm_ms_per_step": warm_ms_step,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "device_status": int(status),
         "roofline": roofline,
         "path_roofline": {"t_roof_ms": t_roof_ms, "frac": t_roof_ms / ms_step, "algorithmic_bytes": work["bytes"],
@@ -352,12 +414,110 @@ def run_ours(args):
         "stage_gbs": {s: stage_bytes[s] / (stage_ms[s] * 1e-3) / 1e9 for s in stage_bytes if stage_ms.get(s, 0) > 0},
         "tokens_per_step": tokens_per_step,
     }
+    if w.name == "decode_round" and world == 1 and not args.no_protocol:
+        del layers
+        torch.cuda.empty_cache()
+        out["decode_protocol"] = decode_protocol(ab, synth, w, dev, stream)
     if world == 1 and not args.no_cpu_baseline:
         _, _, info = cpu_oracle_sample(w)
         out["cpu_baseline"] = info
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def decode_protocol(ab, synth, w, dev, stream):
+    """The decode configuration as a protocol: an untimed prefill eviction of a 32768-token cache down to the budget,
+    then 256 generation steps.  (a) One eviction round every 32 steps with the last 32 queries as observation
+    window, timed per round (8 rounds), with and without the value prior.  (b) Algorithm 1 as printed: evict at
+    every step (one-row score update, selection, compaction in place), 256 steps timed."""
+    import torch
+    B, Hq, Hkv, d, Bud, Br, r = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.budget, w.recent_window, w.obs_window
+    dtc = {"f32": ab.F32, "f16": ab.F16, "bf16": ab.BF16}[w.dtype]
+    n0 = 32768
+    pre = w.scaled(n_ctx=n0, n_total=None, value_prior=True)
+    pp = ab.Params(B, Hq, Hkv, d, n0, r, Br, Bud, dtype=dtc, flags=ab.FLAG_VALUE_PRIOR)
+    q, k, v = synth.make_layer(pre, layer=0, device=dev)
+    ws = ab.alloc_workspace(pp, dev)
+    k0, v0, f0, idx0 = ab.alloc_outputs(pp, dev)
+    ab.ahakv_evict(pp, q, k, v, None, k0, v0, f0, idx0, ws, stream=stream)
+    torch.cuda.synchronize()
+    del q, k, v, ws
+    torch.cuda.empty_cache()
+    new = [synth.make_decode_step(w, t, device=dev) for t in range(256)]
+
+    def rounds(flags):
+        n = Bud + r
+        kc = torch.empty((B, Hkv, n, d), dtype=k0.dtype, device=dev)
+        vc = torch.empty_like(kc)
+        fc = torch.zeros((B, Hkv, n), device=dev)
+        kc[:, :, :Bud], vc[:, :, :Bud], fc[:, :, :Bud] = k0, v0, f0
+        ko, vo, fo, io = ab.alloc_outputs(ab.Params(B, Hq, Hkv, d, n, r, Br, Bud, dtype=dtc), dev)
+        ms = []
+        for rd in range(8):
+            steps = new[rd * r:(rd + 1) * r]
+            qr = torch.cat([x[0] for x in steps], 2).contiguous()
+            kc[:, :, Bud:] = torch.cat([x[1] for x in steps], 2)
+            vc[:, :, Bud:] = torch.cat([x[2] for x in steps], 2)
+            fc[:, :, Bud:] = 0.0
+            p = ab.Params(B, Hq, Hkv, d, n, r, Br, Bud, dtype=dtc, n_total=n0 + (rd + 1) * r, flags=flags)
+            wsr = ab.alloc_workspace(p, dev)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            ab.ahakv_evict(p, qr, kc, vc, fc, ko, vo, fo, io, wsr, stream=stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            assert ab.ahakv_last_device_status(wsr) == ab.OK
+            ms.append(e0.elapsed_time(e1))
+            kc[:, :, :Bud], vc[:, :, :Bud], fc[:, :, :Bud] = ko, vo, fo
+        return ms
+
+    plain = rounds(0)
+    prior = rounds(ab.FLAG_VALUE_PRIOR)
+
+    # evict at every step: the cache holds budget + 1 rows when scored
+    n = Bud + 1
+    kc = torch.empty((B, Hkv, n, d), dtype=k0.dtype, device=dev)
+    vc = torch.empty_like(kc)
+    fc = torch.zeros((B, Hkv, n), device=dev)
+    kc[:, :, :Bud], vc[:, :, :Bud], fc[:, :, :Bud] = k0, v0, f0
+    idx = torch.empty((B, Hkv, Bud), dtype=torch.int32, device=dev)
+    ps = [ab.Params(B, Hq, Hkv, d, n, 1, Br, Bud, dtype=dtc, n_total=n0 + t + 1, flags=0) for t in range(256)]
+    zero = torch.zeros((B, Hkv), device=dev)
+
+    def one(t):
+        qt, kt, vt = new[t]
+        kc[:, :, Bud] = kt[:, :, 0]
+        vc[:, :, Bud] = vt[:, :, 0]
+        fc[:, :, Bud] = zero
+        ab.ahakv_score_step(ps[t], qt, kc, fc, fc, stream=stream)
+        ab.ahakv_select(ps[t], fc, idx, stream=stream)
+        ab.ahakv_compact_inplace(ps[t], kc, vc, fc, idx, stream=stream)
+
+    for t in range(8):
+        one(t)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for t in range(256):
+        one(t)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    per_step_ms = e0.elapsed_time(e1) / 256
+    tokens = B * (Bud + r)
+    return {
+        "prefill": f"untimed eviction of {B} x {n0} tokens to {Bud} rows per KV head (value prior on)",
+        "rounds_ms": plain, "rounds_ms_median": statistics.median(plain), "rounds_ms_min": min(plain),
+        "rounds_tokens_per_s_median": tokens / (statistics.median(plain) * 1e-3),
+        "rounds_value_prior_on_ms": prior, "rounds_value_prior_on_ms_median": statistics.median(prior),
+        "evict_every_step": {"steps": 256, "ms_per_step": per_step_ms,
+                             "includes": "appending the new token's rows (three small torch copies), ahakv_score_step, "
+                                         "ahakv_select, ahakv_compact_inplace",
+                             "tokens_per_s": B * n / (per_step_ms * 1e-3)},
+        "note": "each round allocates its workspace outside the timed region; inputs of a round were written just "
+                "before it, so they may still be in L2 (the cache of one round is 136 MB against 126 MB of L2)",
+    }
 
 
 def main():
