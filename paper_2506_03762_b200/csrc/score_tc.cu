@@ -349,7 +349,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
     }
     if (k_state == 1) {
       const int qb = sc & 1;
-      if (mbar_test(&bars->q_empty[qb], ((sc >> 1) & 1) ^ 1)) {
+      if (mbar_try(&bars->q_empty[qb], ((sc >> 1) & 1) ^ 1)) {
         char* q_smem = tiles + kOffQ + qb * kQBytes;
         mbar_expect_tx(&bars->q_full[qb], q_bytes);
         for (int s = 0; s < n_sub; ++s) {
@@ -362,7 +362,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
       }
     } else if (k_state == 2) {
       const int stage = tc % kKStages, ph = (tc / kKStages) & 1;
-      if (mbar_test(&bars->k_empty[stage], ph ^ 1)) {
+      if (mbar_try(&bars->k_empty[stage], ph ^ 1)) {
         mbar_expect_tx(&bars->k_full[stage], k_bytes);
         char* dst = tiles + kOffK + stage * kKStageBytes;
         for (int s = 0; s < n_sub; ++s) {
@@ -382,7 +382,7 @@ __device__ void producer(const TcArgs& a, const CUtensorMap* qmap, const CUtenso
     }
     if (v_state == 2) {
       const int vs = vc % kVStages;
-      if (mbar_test(&bars->v_empty[vs], ((vc / kVStages) & 1) ^ 1)) {
+      if (mbar_try(&bars->v_empty[vs], ((vc / kVStages) & 1) ^ 1)) {
         mbar_expect_tx(&bars->v_full[vs], n_sub * kVSubBytes);
         char* dst = tiles + kOffV + vs * kVStageBytes;
         for (int s = 0; s < n_sub; ++s)

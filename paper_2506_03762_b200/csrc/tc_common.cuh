@@ -39,17 +39,6 @@ __device__ __forceinline__ bool mbar_try(void* bar, int parity) {
       : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// The same without ever suspending the thread: for a thread that polls several barriers in turn and must not
-// sit on one while another has come free.
-__device__ __forceinline__ bool mbar_test(void* bar, int parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
 // Bounded wait.  Returns false (and records the timeout) if the phase did not complete in time.  The
 // clock is slow to read, so it is looked at only after many failed tries (each of which already sleeps in
 // hardware for a while).
