@@ -140,3 +140,55 @@ def test_evict_every_step_for_64_steps():
         assert torch.equal(f[:, :, :Bud], torch.gather(f_scored, 2, idx.long()))
         evicted_somewhere_other_than_the_end += int((gi[..., 0] != 0).sum() + (gi[..., Bud // 2] != Bud // 2).sum())
     assert evicted_somewhere_other_than_the_end > 0                 # the moves were real ones
+
+
+def test_generation_steps_replay_from_a_cuda_graph():
+    """The three calls of a generation step make no allocation, no synchronisation and no host-side decision that
+    depends on device data, so a loop of steps can be captured once and replayed: eight steps captured in a CUDA
+    graph leave the cache, the scores and the kept indices bit-identical to the same eight steps launched one by
+    one.  (Every entry point is called once before the capture: first calls set function attributes.)"""
+    from paper_2506_03762_b200 import binding as ab
+    B, Hq, Hkv, d, Bud, Br, steps, N0 = 2, 8, 2, 128, 512, 32, 8, 9000
+    n = Bud + 1
+    g = torch.Generator().manual_seed(762)
+    dt = torch.float16
+    k0 = torch.zeros((B, Hkv, n, d), dtype=dt, device=DEV)
+    v0 = torch.zeros_like(k0)
+    k0[:, :, :Bud] = torch.randn((B, Hkv, Bud, d), generator=g).to(dt).to(DEV)
+    v0[:, :, :Bud] = torch.randn((B, Hkv, Bud, d), generator=g).to(dt).to(DEV)
+    f0 = torch.zeros((B, Hkv, n), device=DEV)
+    f0[:, :, :Bud] = (torch.rand((B, Hkv, Bud), generator=g) * 0.02).to(DEV)
+    new = [(torch.randn((B, Hq, 1, d), generator=g).to(dt).to(DEV), torch.randn((B, Hkv, d), generator=g).to(dt).to(DEV),
+            torch.randn((B, Hkv, d), generator=g).to(dt).to(DEV)) for _ in range(steps)]
+    ps = [ab.Params(B, Hq, Hkv, d, n, 1, Br, Bud, dtype=ab.F16, n_total=N0 + t + 1, flags=0) for t in range(steps)]
+    zero = torch.zeros((B, Hkv), device=DEV)
+
+    def run(k, v, f, idx, stream):
+        for t in range(steps):
+            q_t, k_t, v_t = new[t]
+            k[:, :, Bud] = k_t
+            v[:, :, Bud] = v_t
+            f[:, :, Bud] = zero
+            ab.ahakv_score_step(ps[t], q_t, k, f, f, stream=stream)
+            ab.ahakv_select(ps[t], f, idx, stream=stream)
+            ab.ahakv_compact_inplace(ps[t], k, v, f, idx, stream=stream)
+
+    ke, ve, fe = k0.clone(), v0.clone(), f0.clone()
+    ie = torch.empty((B, Hkv, Bud), dtype=torch.int32, device=DEV)
+    run(ke, ve, fe, ie, None)
+    torch.cuda.synchronize()
+
+    kg, vg, fg = k0.clone(), v0.clone(), f0.clone()
+    ig = torch.empty_like(ie)
+    s = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(graph, stream=s):
+            run(kg, vg, fg, ig, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    for _ in range(2):                       # the replay starts from the same state each time
+        kg.copy_(k0); vg.copy_(v0); fg.copy_(f0)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(kg[:, :, :Bud], ke[:, :, :Bud]) and torch.equal(vg[:, :, :Bud], ve[:, :, :Bud])
+        assert torch.equal(fg[:, :, :Bud], fe[:, :, :Bud]) and torch.equal(ig, ie)
