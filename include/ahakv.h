@@ -138,6 +138,28 @@ ahakv_status ahakv_score_step(const ahakv_params* p, const void* q_t, const void
 ahakv_status ahakv_compact_inplace(const ahakv_params* p, void* k, void* v, float* score, const int32_t* kept_idx,
                                    ahakv_stream_t stream);
 
+/* One generation step on a cache kept as slots (Algorithm 1, Generation, with K <- K_S, V <- V_S done by bookkeeping
+ * instead of by moving rows).  Attention does not depend on the order of the cached rows, and Algorithm 1 uses a
+ * token's position only to protect the most recent ones, so the cache of a (sequence, KV head) can be a set of
+ * budget + 1 slots with a table of positions: the evicted token's slot is where the next token is written, and no
+ * row is ever moved.  Per (sequence, KV head), in one kernel: the new token's key and value rows (k_t, v_t:
+ * [B,Hkv,1,d], dense) are copied into slot free_slot[b,h]; the one new query per head (q_t: [B,Hq,1,d]) is scored
+ * against all budget + 1 slots exactly as ahakv_score_step does (lambda of Eq. 12 from p->n_total, the number of
+ * tokens so far with the new one); score ([B,Hkv,budget+1] float32) becomes F_t = SGsoftmax(A_t) + F_{t-1} in
+ * place, the new token starting from zero; pos ([B,Hkv,budget+1] int32, the position of the token in each slot)
+ * gets p->n_total - 1 for the new token; and of the slots whose position is below p->n_total - recent_window (the
+ * recent window is the last recent_window positions, the new token's included, and is never evicted, so those
+ * tokens are all in the cache) the one with the smallest score -- of equal scores the most recent token, which is
+ * the token ahakv_select drops when it keeps the lowest indices among ties -- is declared free: pos = -1 there and
+ * free_slot[b,h] = its index.  The result is the cache ahakv_score_step + ahakv_select + ahakv_compact_inplace
+ * leave, up to the order of the rows.
+ * p->n_ctx must be budget + 1 and p->obs_window 1; the limits of ahakv_score_step apply (AHAKV_ERR_UNSUPPORTED
+ * otherwise).  k, v: [B,Hkv,budget+1,d] with the strides of p.  A free_slot entry outside [0, budget] leaves that
+ * head untouched; a position table in which no slot lies outside the recent window sets free_slot[b,h] = -1.  To
+ * start from a cache of budget rows in order: slots 0 .. budget-1 with pos = their positions, free_slot = budget. */
+ahakv_status ahakv_step_slots(const ahakv_params* p, const void* q_t, const void* k_t, const void* v_t, void* k, void* v,
+                              float* score, int32_t* pos, int32_t* free_slot, ahakv_stream_t stream);
+
 /* Row entropy of the scaled softmax (Section 4.2, Eq. 6): H_i = - sum_j a_ij ln a_ij (natural log) for every
  * observation row of every query head, with a_ij exactly as in ahakv_score (mask, lambda from scale_mode).  A
  * diagnostic: Eq. 10 predicts E[H_i] = ln i - lambda^2 d / 2, and Eq. 12 picks lambda so that this is ln(budget).

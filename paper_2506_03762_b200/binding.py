@@ -92,6 +92,7 @@ SIGNATURES = {
     "ahakv_score_full_causal": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_score_step": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_compact_inplace": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp]),
+    "ahakv_step_slots": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_entropy_workspace_bytes": (_sz, [_PP]),
     "ahakv_row_entropy": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_select": (ctypes.c_int, [_PP, _vp, _vp, _vp, _sz, _vp]),
@@ -218,6 +219,15 @@ def ahakv_compact_inplace(p: Params, k, v, score, kept_idx, stream=None, check: 
     st = lib().ahakv_compact_inplace(ctypes.byref(cp), _ptr(k), _ptr(v), _ptr(score), _ptr(kept_idx), _stream(stream))
     if check:
         _raise(st, "ahakv_compact_inplace")
+    return st
+
+
+def ahakv_step_slots(p: Params, q_t, k_t, v_t, k, v, score, pos, free_slot, stream=None, check: bool = True) -> int:
+    cp = p.c()
+    st = lib().ahakv_step_slots(ctypes.byref(cp), _ptr(q_t), _ptr(k_t), _ptr(v_t), _ptr(k), _ptr(v), _ptr(score),
+                                _ptr(pos), _ptr(free_slot), _stream(stream))
+    if check:
+        _raise(st, "ahakv_step_slots")
     return st
 
 

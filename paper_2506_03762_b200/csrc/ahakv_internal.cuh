@@ -60,6 +60,8 @@ void score_tc_test_hooks(long long wait_ns, int withhold);   // see ahakv_test_s
 // The generation phase one token at a time (decode.cu): the score update of one new query per head without
 // scratch memory, and compaction in place.
 bool step_score_fits(const Plan& pl);
+ahakv_status launch_step_slots(const Plan& pl, const void* q, const void* k_new, const void* v_new, void* k, void* v,
+                               float* score, int32_t* pos, int32_t* free_slot, int new_pos, cudaStream_t st);
 ahakv_status launch_step_score(const Plan& pl, const void* q, const void* k, const float* prev, float* score,
                                cudaStream_t st);
 ahakv_status launch_compact_inplace(const Plan& pl, void* k, void* v, float* score, const int32_t* kept_idx,

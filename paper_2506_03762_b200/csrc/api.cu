@@ -279,6 +279,21 @@ ahakv_status ahakv_score_step(const ahakv_params* p, const void* q_t, const void
   return launch_step_score(pl, q_t, k, score_prev, score, (cudaStream_t)stream);
 }
 
+ahakv_status ahakv_step_slots(const ahakv_params* p, const void* q_t, const void* k_t, const void* v_t, void* k, void* v,
+                              float* score, int32_t* pos, int32_t* free_slot, ahakv_stream_t stream) {
+  Plan pl;
+  ahakv_status rc = make_plan(p, &pl);
+  if (rc) return rc;
+  if (pl.r != 1 || pl.n != pl.Bud + 1) return AHAKV_ERR_INVALID_ARG;
+  if (!q_t || !k_t || !v_t || !k || !v || !score || !pos || !free_slot || !aligned16(q_t) || !aligned16(k_t) ||
+      !aligned16(v_t) || !aligned16(k) || !aligned16(v) || ((uintptr_t)score & 3) || ((uintptr_t)pos & 3) ||
+      ((uintptr_t)free_slot & 3))
+    return AHAKV_ERR_INVALID_ARG;
+  if (pl.n_total - 1 > 0x7ffffffe) return AHAKV_ERR_INVALID_ARG;
+  if ((pl.flags & AHAKV_FLAG_VALUE_PRIOR) || !step_score_fits(pl)) return AHAKV_ERR_UNSUPPORTED;
+  return launch_step_slots(pl, q_t, k_t, v_t, k, v, score, pos, free_slot, (int)(pl.n_total - 1), (cudaStream_t)stream);
+}
+
 ahakv_status ahakv_compact_inplace(const ahakv_params* p, void* k, void* v, float* score, const int32_t* kept_idx,
                                    ahakv_stream_t stream) {
   Plan pl;

@@ -15,11 +15,12 @@
 #include <type_traits>
 
 #include "ahakv_internal.cuh"
+#include "select_common.cuh"
 
 namespace ahakv {
 namespace {
 
-constexpr int kStepThreads = 256;
+constexpr int kStepThreads = 512;
 constexpr int kStepMaxG = 16;                  // query heads per KV head the step kernel takes
 constexpr size_t kStepMaxLogitBytes = 160 * 1024;   // 40960 logits
 
@@ -41,19 +42,15 @@ __device__ __forceinline__ float block_reduce(float x, float* red) {
   return r;
 }
 
-// LANES threads share a key row (16 bytes each); kG query heads.
+// The G x n logits of one (sequence, KV head), in log2 units, into shared memory.  LANES threads share a key row
+// (16 bytes each); kG query heads.
 template <typename T, int D, int kG>
-__global__ void __launch_bounds__(kStepThreads) step_score_kernel(const T* __restrict__ q, const T* __restrict__ k,
-                                                                  const float* __restrict__ prev,
-                                                                  float* __restrict__ score, const Shape pl,
-                                                                  const double c_row) {
+__device__ __forceinline__ void step_logits(const T* __restrict__ q, const T* __restrict__ k, const Shape& pl, int b,
+                                            int h, Acc<T> c, float* logit) {
   using A = Acc<T>;
   constexpr int V = Vec16<T>::N, LANES = D / V, KEYS_PER_WARP = 32 / LANES;
-  extern __shared__ __align__(16) float logit[];                 // [kG][n]
-  __shared__ float red[kStepThreads / 32];
-  const int unit = blockIdx.x, b = unit / pl.Hkv, h = unit % pl.Hkv, n = pl.n;
+  const int n = pl.n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, sub = lane % LANES, which = lane / LANES;
-  const A c = (A)c_row;
 
   // this lane's slice of each of the group's queries
   float qreg[kG][V];
@@ -89,9 +86,11 @@ __global__ void __launch_bounds__(kStepThreads) step_score_kernel(const T* __res
     }
   }
   __syncthreads();
+}
 
-  // per query head: shift and normaliser, then 2^{x - M} / (G Z) in place
-  const float inv_g = pl.group_max ? 1.f : 1.f / (float)kG;
+// Per query head: shift and normaliser, then 2^{x - M} / (G Z) in place of the logits.
+template <int kG>
+__device__ __forceinline__ void step_weights(float* logit, int n, float inv_g, float* red) {
   for (int g = 0; g < kG; ++g) {
     float* x = logit + g * n;
     float m = -INFINITY;
@@ -108,12 +107,106 @@ __global__ void __launch_bounds__(kStepThreads) step_score_kernel(const T* __res
     for (int j = threadIdx.x; j < n; j += kStepThreads) x[j] *= w;
   }
   __syncthreads();
-  for (int j = threadIdx.x; j < n; j += kStepThreads) {
-    float s = logit[j];
+}
+
+// Token j's share of the step: the weights of the group's heads pooled.
+template <int kG>
+__device__ __forceinline__ float step_pooled(const float* logit, int n, int j, int group_max) {
+  float s = logit[j];
 #pragma unroll
-    for (int g = 1; g < kG; ++g) s = pl.group_max ? fmaxf(s, logit[g * n + j]) : s + logit[g * n + j];
+  for (int g = 1; g < kG; ++g) s = group_max ? fmaxf(s, logit[g * n + j]) : s + logit[g * n + j];
+  return s;
+}
+
+template <typename T, int D, int kG>
+__global__ void __launch_bounds__(kStepThreads) step_score_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                                  const float* __restrict__ prev,
+                                                                  float* __restrict__ score, const Shape pl,
+                                                                  const double c_row) {
+  extern __shared__ __align__(16) float logit[];                 // [kG][n]
+  __shared__ float red[kStepThreads / 32];
+  const int unit = blockIdx.x, b = unit / pl.Hkv, h = unit % pl.Hkv, n = pl.n;
+  step_logits<T, D, kG>(q, k, pl, b, h, (Acc<T>)c_row, logit);
+  step_weights<kG>(logit, n, pl.group_max ? 1.f : 1.f / (float)kG, red);
+  for (int j = threadIdx.x; j < n; j += kStepThreads) {
+    float s = step_pooled<kG>(logit, n, j, pl.group_max);
     if (prev) s = __fadd_rn(s, prev[(size_t)unit * n + j]);
     score[(size_t)unit * n + j] = s;
+  }
+}
+
+// One generation step on a cache kept as slots (no row ever moves): the new token's key and value rows go into the
+// free slot of the (sequence, KV head), the one new query per head is scored against every slot, the score is
+// updated in place, and the slot with the smallest score outside the recent window -- of equal scores the most recent
+// token -- is declared free for the next step.  `pos` holds the logical position of the token in each slot; the
+// recent window is the recent_window largest positions, the new token's included.
+template <typename T, int D, int kG>
+__global__ void __launch_bounds__(kStepThreads) step_slots_kernel(const T* __restrict__ q, const T* __restrict__ k_new,
+                                                                  const T* __restrict__ v_new, T* __restrict__ k,
+                                                                  T* __restrict__ v, float* __restrict__ score,
+                                                                  int32_t* __restrict__ pos, int32_t* __restrict__ free_slot,
+                                                                  const Shape pl, const double c_row, const int new_pos) {
+  extern __shared__ __align__(16) float logit[];                 // [kG][n]
+  __shared__ float red[kStepThreads / 32];
+  __shared__ unsigned long long best[kStepThreads / 32];
+  constexpr int V = Vec16<T>::N, LANES = D / V;
+  const int unit = blockIdx.x, b = unit / pl.Hkv, h = unit % pl.Hkv, n = pl.n;
+  float* sc = score + (size_t)unit * n;
+  int32_t* ps = pos + (size_t)unit * n;
+  const int slot = free_slot[unit];
+  if (slot < 0 || slot >= n) return;                             // the caller's table is broken: touch nothing
+  // the new token moves in
+  if (threadIdx.x < 2 * LANES) {
+    const int sub = threadIdx.x % LANES;
+    const bool is_v = threadIdx.x >= LANES;
+    const T* src = (is_v ? v_new : k_new) + ((long long)b * pl.Hkv + h) * D + sub * V;
+    T* dst = is_v ? v + (long long)b * pl.vs[0] + (long long)h * pl.vs[1] + (long long)slot * pl.vs[2] + sub * V
+                  : k + (long long)b * pl.ks[0] + (long long)h * pl.ks[1] + (long long)slot * pl.ks[2] + sub * V;
+    *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
+  }
+  __syncthreads();                                               // the row is read back by other threads below
+  step_logits<T, D, kG>(q, k, pl, b, h, (Acc<T>)c_row, logit);
+  step_weights<kG>(logit, n, pl.group_max ? 1.f : 1.f / (float)kG, red);
+  // F_t = SGsoftmax(A_t) + F_{t-1}, and the candidate to leave: smallest score, then largest position
+  const int oldest_protected = new_pos - pl.Br + 1;             // positions from here on are the recent window
+  unsigned long long mine = ~0ull;
+  for (int j = threadIdx.x; j < n; j += kStepThreads) {
+    float s = step_pooled<kG>(logit, n, j, pl.group_max);
+    const int pj = j == slot ? new_pos : ps[j];
+    if (j != slot) s = __fadd_rn(s, sc[j]);                      // a new token starts at zero
+    sc[j] = s;
+    if (pj < oldest_protected) {
+      // ascending in (score, -position): the position is below 2^31, so ~pj orders it downwards within 32 bits
+      const unsigned long long key = ((unsigned long long)order_key(s) << 32) | (unsigned)(0x7fffffff - pj);
+      if (key < mine) mine = key;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    const unsigned long long y = __shfl_xor_sync(0xffffffffu, mine, o);
+    if (y < mine) mine = y;
+  }
+  if ((threadIdx.x & 31) == 0) best[threadIdx.x >> 5] = mine;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long m = best[0];
+    for (int w = 1; w < kStepThreads / 32; ++w) if (best[w] < m) m = best[w];
+    best[0] = m;
+  }
+  __syncthreads();
+  const unsigned long long win = best[0];
+  if (win == ~0ull) {                                            // no slot outside the recent window: a broken position table
+    if (threadIdx.x == 0) free_slot[unit] = -1;
+    return;
+  }
+  const int win_pos = 0x7fffffff - (int)(unsigned)(win & 0xffffffffu);
+  for (int j = threadIdx.x; j < n; j += kStepThreads) {
+    const int pj = j == slot ? new_pos : ps[j];
+    if (j == slot) ps[j] = new_pos;
+    if (pj == win_pos) {                                         // positions are distinct: exactly one slot
+      ps[j] = -1;
+      free_slot[unit] = j;
+    }
   }
 }
 
@@ -136,6 +229,46 @@ ahakv_status launch_step_as(const Plan& pl, const void* q, const void* k, const 
                                                                       pl.lambda[0] * 1.4426950408889634);
   count_launch();
   return cuda_ok(cudaGetLastError());
+}
+
+template <typename T, int D, int kG>
+ahakv_status launch_slots_as(const Plan& pl, const void* q, const void* k_new, const void* v_new, void* k, void* v,
+                             float* score, int32_t* pos, int32_t* free_slot, int new_pos, cudaStream_t st) {
+  const size_t smem = (size_t)kG * pl.n * sizeof(float);
+  constexpr int kMaxDevices = 64;
+  static size_t configured[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return AHAKV_ERR_CUDA;
+  if (smem > 40 * 1024 && configured[dev] < kStepMaxLogitBytes) {
+    if (cudaFuncSetAttribute(step_slots_kernel<T, D, kG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kStepMaxLogitBytes) != cudaSuccess)
+      return AHAKV_ERR_CUDA;
+    configured[dev] = kStepMaxLogitBytes;
+  }
+  const Shape& shape = pl;
+  step_slots_kernel<T, D, kG><<<pl.B * pl.Hkv, kStepThreads, smem, st>>>(
+      (const T*)q, (const T*)k_new, (const T*)v_new, (T*)k, (T*)v, score, pos, free_slot, shape,
+      pl.lambda[0] * 1.4426950408889634, new_pos);
+  count_launch();
+  return cuda_ok(cudaGetLastError());
+}
+
+template <typename T, int D>
+ahakv_status launch_slots_g(const Plan& pl, const void* q, const void* k_new, const void* v_new, void* k, void* v,
+                            float* score, int32_t* pos, int32_t* free_slot, int new_pos, cudaStream_t st) {
+  switch (pl.G) {
+    case 1: return launch_slots_as<T, D, 1>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case 2: return launch_slots_as<T, D, 2>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case 3: return launch_slots_as<T, D, 3>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case 4: return launch_slots_as<T, D, 4>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case 5: return launch_slots_as<T, D, 5>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case 6: return launch_slots_as<T, D, 6>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case 7: return launch_slots_as<T, D, 7>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case 8: return launch_slots_as<T, D, 8>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case 12: return launch_slots_as<T, D, 12>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case 16: return launch_slots_as<T, D, 16>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    default: return AHAKV_ERR_UNSUPPORTED;
+  }
 }
 
 template <typename T, int D>
@@ -222,6 +355,22 @@ ahakv_status launch_step_score(const Plan& pl, const void* q, const void* k, con
     case AHAKV_F16: return d64 ? launch_step_g<__half, 64>(pl, q, k, prev, score, st) : launch_step_g<__half, 128>(pl, q, k, prev, score, st);
     default: return d64 ? launch_step_g<__nv_bfloat16, 64>(pl, q, k, prev, score, st)
                         : launch_step_g<__nv_bfloat16, 128>(pl, q, k, prev, score, st);
+  }
+}
+
+ahakv_status launch_step_slots(const Plan& pl, const void* q, const void* k_new, const void* v_new, void* k, void* v,
+                               float* score, int32_t* pos, int32_t* free_slot, int new_pos, cudaStream_t st) {
+  const bool d64 = pl.d == 64;
+  switch (pl.dtype) {
+    case AHAKV_F32:
+      return d64 ? launch_slots_g<float, 64>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st)
+                 : launch_slots_g<float, 128>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    case AHAKV_F16:
+      return d64 ? launch_slots_g<__half, 64>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st)
+                 : launch_slots_g<__half, 128>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
+    default:
+      return d64 ? launch_slots_g<__nv_bfloat16, 64>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st)
+                 : launch_slots_g<__nv_bfloat16, 128>(pl, q, k_new, v_new, k, v, score, pos, free_slot, new_pos, st);
   }
 }
 

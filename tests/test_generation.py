@@ -192,3 +192,68 @@ def test_generation_steps_replay_from_a_cuda_graph():
         torch.cuda.synchronize()
         assert torch.equal(kg[:, :, :Bud], ke[:, :, :Bud]) and torch.equal(vg[:, :, :Bud], ve[:, :, :Bud])
         assert torch.equal(fg[:, :, :Bud], fe[:, :, :Bud]) and torch.equal(ig, ie)
+
+
+@pytest.mark.parametrize("dtype_name,Hq,Hkv,d", [("BF16", 8, 2, 128), ("F16", 4, 4, 64), ("F32", 6, 2, 128)])
+def test_step_slots_for_48_steps(dtype_name, Hq, Hkv, d):
+    """Generation on a cache kept as slots: nothing moves, the evicted token's slot takes the next token.  Every step
+    is checked against the oracle run on the same cache put in order of position (scores within tolerance, the kept
+    set equal outside the tolerance band), and the bookkeeping exactly: the new rows sit byte for byte in the slot that
+    was free, no other slot changed, the position table and the free slot say which token left."""
+    from paper_2506_03762_b200 import binding as ab
+    from tests import parity
+    B, Bud, Br, steps, N0 = 2, 192, 12, 48, 7000
+    n = Bud + 1
+    dtc = getattr(ab, dtype_name)
+    dt = {"F32": torch.float32, "F16": torch.float16, "BF16": torch.bfloat16}[dtype_name]
+    g = torch.Generator().manual_seed(1200 + d + Hq)
+    k = torch.zeros((B, Hkv, n, d), dtype=dt, device=DEV)
+    v = torch.zeros_like(k)
+    k[:, :, :Bud] = torch.randn((B, Hkv, Bud, d), generator=g).to(dt).to(DEV)
+    v[:, :, :Bud] = torch.randn((B, Hkv, Bud, d), generator=g).to(dt).to(DEV)
+    f = torch.zeros((B, Hkv, n), device=DEV)
+    f[:, :, :Bud] = (torch.rand((B, Hkv, Bud), generator=g) * 0.02).to(DEV)
+    # positions of the cached tokens: scattered, in order, below the recent window; then the window itself
+    old = torch.sort(torch.randperm(N0 - Br, generator=g)[:Bud - Br]).values
+    pos0 = torch.cat([old, torch.arange(N0 - Br, N0)]).to(torch.int32)
+    pos = torch.full((B, Hkv, n), -1, dtype=torch.int32, device=DEV)
+    pos[:, :, :Bud] = pos0.to(DEV)
+    # the slots are in no particular order: shuffle them, per head
+    for b in range(B):
+        for h in range(Hkv):
+            perm = torch.randperm(n, generator=g).to(DEV)
+            k[b, h], v[b, h], f[b, h], pos[b, h] = k[b, h][perm].clone(), v[b, h][perm].clone(), f[b, h][perm].clone(), pos[b, h][perm].clone()
+    free = (pos == -1).int().argmax(dim=2).to(torch.int32).contiguous()
+    for t in range(steps):
+        p = ab.Params(B, Hq, Hkv, d, n, 1, Br, Bud, dtype=dtc, n_total=N0 + t + 1, flags=0)
+        new_pos = N0 + t
+        q_t = torch.randn((B, Hq, 1, d), generator=g).to(dt).to(DEV)
+        k_t = torch.randn((B, Hkv, 1, d), generator=g).to(dt).to(DEV)
+        v_t = torch.randn((B, Hkv, 1, d), generator=g).to(dt).to(DEV)
+        k0, v0, f0, pos_before, free_before = k.clone(), v.clone(), f.clone(), pos.clone(), free.clone()
+        ab.ahakv_step_slots(p, q_t, k_t, v_t, k, v, f, pos, free)
+        torch.cuda.synchronize()
+        # bookkeeping
+        fb = free_before.long()[:, :, None]
+        pos_full = pos_before.clone().scatter_(2, fb, torch.full_like(fb, new_pos, dtype=torch.int32))
+        k_full = k0.clone().scatter_(2, fb[..., None].expand(B, Hkv, 1, d), k_t)
+        v_full = v0.clone().scatter_(2, fb[..., None].expand(B, Hkv, 1, d), v_t)
+        assert torch.equal(k, k_full) and torch.equal(v, v_full), f"step {t}: rows"
+        fa = free.long()[:, :, None]
+        assert bool(((free >= 0) & (free < n)).all())
+        assert torch.equal(pos, pos_full.clone().scatter_(2, fa, torch.full_like(fa, -1, dtype=torch.int32))), f"step {t}: positions"
+        assert bool((pos_full.gather(2, fa) < new_pos - Br + 1).all()), "a token of the recent window left"
+        # the oracle on the cache in order of position (the new token last, with score zero)
+        order = torch.argsort(pos_full, dim=2)
+        ko = k_full.gather(2, order[..., None].expand(B, Hkv, n, d))
+        vo = v_full.gather(2, order[..., None].expand(B, Hkv, n, d))
+        f_prev = f0.clone().scatter_(2, fb, torch.zeros_like(fb, dtype=torch.float32)).gather(2, order)
+        op = parity.oracle_params(p)
+        ref = orc.evict(op, synth.to_numpy(q_t), synth.to_numpy(ko), synth.to_numpy(vo), f_prev.double().cpu().numpy())
+        parity.assert_scores_close(p, f.gather(2, order).cpu().numpy(), ref["score"], f"step {t} score")
+        rank_of_slot = torch.argsort(order, dim=2)                     # slot -> index in position order
+        left = rank_of_slot.gather(2, fa)[:, :, 0].cpu().numpy()
+        for b in range(B):
+            for h in range(Hkv):
+                kept = np.array([j for j in range(n) if j != left[b, h]], dtype=np.int32)
+                parity.assert_kept_valid(p, kept, ref["kept_idx"][b, h], ref["score"][b, h])
