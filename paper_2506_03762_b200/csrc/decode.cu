@@ -2,11 +2,15 @@
 // then S = TopK(F_t, B_s) U recent B_r and K <- K_S, V <- V_S before the next token).
 //
 // step_score_kernel: one CTA per (sequence, KV head).  The G query rows of the group (one new query per head)
-//   against the n cached keys is a matrix-vector product, bound by reading K once: half a warp (or a quarter,
-//   or a whole one, by row size) reads one key row with 16-byte loads, every lane keeps its slice of the G
-//   queries in registers, and the partial dot products meet by shuffle.  The G x n logits stay in shared memory;
-//   row maxima and sums are block reductions in a fixed order; the new score is written in one more sweep.
+//   against the n cached keys is a matrix-vector product, bound by reading K once.  16-bit inputs: warp-level
+//   m16n8k16 products, the heads on the rows and eight keys on the columns (step_logits_mma).  float32 inputs:
+//   half a warp (or a quarter, by row size) reads one key row with 16-byte loads, every lane keeps its slice of
+//   the G queries in registers, and the partial dot products meet by shuffle.  The G x n logits stay in shared
+//   memory; row maxima and sums are block reductions in a fixed order; the new score is written in one more sweep.
 //   No scratch memory, no second read of K.
+//
+// step_slots_kernel: the same, for a cache kept as slots: it also copies the new token's rows into the free slot
+//   and names the slot that becomes free (smallest score outside the recent window).
 //
 // compact_inplace_kernel: one CTA per (sequence, KV head).  kept_idx is ascending, so row t of the result comes
 //   from row kept_idx[t] >= t: rows before the first evicted index do not move at all, and the others move in
@@ -88,6 +92,102 @@ __device__ __forceinline__ void step_logits(const T* __restrict__ q, const T* __
   __syncthreads();
 }
 
+// The same logits for 16-bit inputs on the warp-level tensor-core instruction: a G x n by d product is far too
+// thin for the tensor memory path, but the FP32 multiply-add loop above spends forty-odd instructions a key on
+// conversions and shuffle reductions, and mma.sync m16n8k16 (heads on the 16 rows, 8 keys on the columns, FP32
+// accumulation of exact products) spends three.  The sum over d does not care in which order d is walked, so each
+// thread takes one contiguous quarter of a row -- of its query head's row for the A operand, of its key's row for the
+// B operand -- and hands its 32-bit words to the instruction in pairs: the k-slices the four threads of a group
+// present side by side are then the same permutation of d for A and for B.
+template <typename T> struct Mma16816;
+template <> struct Mma16816<__half> {
+  static __device__ __forceinline__ void run(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  }
+};
+template <> struct Mma16816<__nv_bfloat16> {
+  static __device__ __forceinline__ void run(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                             uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  }
+};
+
+template <typename T, int D, int kG>
+__device__ __forceinline__ void step_logits_mma(const T* __restrict__ q, const T* __restrict__ k, const Shape& pl, int b,
+                                                int h, float c, float* logit) {
+  constexpr int CH = D / 4, W = CH / 2, Q4 = CH / 8;           // a thread's quarter row: elements, 32-bit words, 16-byte loads
+  constexpr int kSteps = D / 16, kUnroll = 4, kWarps = kStepThreads / 32;
+  const int n = pl.n;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, grp = lane >> 2, tig = lane & 3;
+
+  // A: head `grp` (and `grp + 8` when there are more than eight) of the group's queries, this thread's quarter
+  uint32_t qa[W], qb[W];
+#pragma unroll
+  for (int t = 0; t < W; ++t) { qa[t] = 0u; qb[t] = 0u; }
+  if (grp < kG) {
+    const T* row = q + (long long)b * pl.qs[0] + (long long)(h * pl.G + grp) * pl.qs[1] + CH * tig;
+#pragma unroll
+    for (int t = 0; t < Q4; ++t) {
+      const uint4 u = *reinterpret_cast<const uint4*>(row + 8 * t);
+      qa[4 * t] = u.x; qa[4 * t + 1] = u.y; qa[4 * t + 2] = u.z; qa[4 * t + 3] = u.w;
+    }
+  }
+  if (kG > 8 && grp + 8 < kG) {
+    const T* row = q + (long long)b * pl.qs[0] + (long long)(h * pl.G + grp + 8) * pl.qs[1] + CH * tig;
+#pragma unroll
+    for (int t = 0; t < Q4; ++t) {
+      const uint4 u = *reinterpret_cast<const uint4*>(row + 8 * t);
+      qb[4 * t] = u.x; qb[4 * t + 1] = u.y; qb[4 * t + 2] = u.z; qb[4 * t + 3] = u.w;
+    }
+  }
+  const T* kbase = k + (long long)b * pl.ks[0] + (long long)h * pl.ks[1] + CH * tig;
+  const int n_blocks = (n + 7) / 8;
+  for (int blk0 = warp; blk0 < n_blocks; blk0 += kWarps * kUnroll) {
+    uint4 raw[kUnroll][Q4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int j = (blk0 + u * kWarps) * 8 + grp;               // this thread's key in block u
+#pragma unroll
+      for (int t = 0; t < Q4; ++t)
+        raw[u][t] = j < n ? *reinterpret_cast<const uint4*>(kbase + (long long)j * pl.ks[2] + 8 * t) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int j0 = (blk0 + u * kWarps) * 8;
+      if (j0 >= n) break;                                        // uniform over the warp
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int t = 0; t < Q4; ++t) {
+        const uint32_t w[4] = {raw[u][t].x, raw[u][t].y, raw[u][t].z, raw[u][t].w};
+        // two k-steps a 16-byte load: words (0, 1) and (2, 3)
+        Mma16816<T>::run(acc, qa[4 * t], qb[4 * t], qa[4 * t + 1], qb[4 * t + 1], w[0], w[1]);
+        Mma16816<T>::run(acc, qa[4 * t + 2], qb[4 * t + 2], qa[4 * t + 3], qb[4 * t + 3], w[2], w[3]);
+      }
+      static_assert(kSteps == 2 * Q4, "two k-steps per 16-byte load");
+      const int j = j0 + 2 * tig;
+      if (grp < kG) {
+        if (j < n) logit[grp * n + j] = acc[0] * c;
+        if (j + 1 < n) logit[grp * n + j + 1] = acc[1] * c;
+      }
+      if (kG > 8 && grp + 8 < kG) {
+        if (j < n) logit[(grp + 8) * n + j] = acc[2] * c;
+        if (j + 1 < n) logit[(grp + 8) * n + j + 1] = acc[3] * c;
+      }
+    }
+  }
+  __syncthreads();
+}
+
+template <typename T, int D, int kG>
+__device__ __forceinline__ void step_logits_any(const T* __restrict__ q, const T* __restrict__ k, const Shape& pl, int b,
+                                                int h, double c_row, float* logit) {
+  if constexpr (std::is_same<T, float>::value) step_logits<T, D, kG>(q, k, pl, b, h, (Acc<T>)c_row, logit);
+  else step_logits_mma<T, D, kG>(q, k, pl, b, h, (float)c_row, logit);
+}
+
 // Per query head: shift and normaliser, then 2^{x - M} / (G Z) in place of the logits.
 template <int kG>
 __device__ __forceinline__ void step_weights(float* logit, int n, float inv_g, float* red) {
@@ -126,7 +226,7 @@ __global__ void __launch_bounds__(kStepThreads) step_score_kernel(const T* __res
   extern __shared__ __align__(16) float logit[];                 // [kG][n]
   __shared__ float red[kStepThreads / 32];
   const int unit = blockIdx.x, b = unit / pl.Hkv, h = unit % pl.Hkv, n = pl.n;
-  step_logits<T, D, kG>(q, k, pl, b, h, (Acc<T>)c_row, logit);
+  step_logits_any<T, D, kG>(q, k, pl, b, h, c_row, logit);
   step_weights<kG>(logit, n, pl.group_max ? 1.f : 1.f / (float)kG, red);
   for (int j = threadIdx.x; j < n; j += kStepThreads) {
     float s = step_pooled<kG>(logit, n, j, pl.group_max);
@@ -165,7 +265,7 @@ __global__ void __launch_bounds__(kStepThreads) step_slots_kernel(const T* __res
     *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
   }
   __syncthreads();                                               // the row is read back by other threads below
-  step_logits<T, D, kG>(q, k, pl, b, h, (Acc<T>)c_row, logit);
+  step_logits_any<T, D, kG>(q, k, pl, b, h, c_row, logit);
   step_weights<kG>(logit, n, pl.group_max ? 1.f : 1.f / (float)kG, red);
   // F_t = SGsoftmax(A_t) + F_{t-1}, and the candidate to leave: smallest score, then largest position
   const int oldest_protected = new_pos - pl.Br + 1;             // positions from here on are the recent window

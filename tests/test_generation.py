@@ -23,6 +23,9 @@ def _dt(ab, dtype):
     (1, 6, 2, 64, 300, "F32", 0),              # three query heads a group, float32 at 1e-5
     (3, 7, 1, 64, 515, "F16", 4),              # seven heads a group pooled by maximum
     (1, 1, 1, 128, 1, "F16", 0),               # a single cached token
+    (1, 12, 1, 128, 1003, "BF16", 0),          # twelve heads a group: both halves of the 16-row product
+    (2, 16, 1, 64, 2044, "F16", 0),            # sixteen heads, 64-wide rows, a ragged last block of keys
+    (1, 16, 2, 64, 333, "BF16", 4),            # eight heads a group pooled by maximum
 ])
 def test_score_step_matches_the_oracle_and_the_general_path(B, Hq, Hkv, d, n, dtype_name, flags):
     from paper_2506_03762_b200 import binding as ab
