@@ -43,7 +43,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling small cases)")
     ap.add_argument("--capture", action="store_true",
-                    help="profiler-friendly run: exactly --warmup and --steps calls of ahakv_evict, nothing else")
+                    help="profiler-friendly run: exactly --warmup and --steps calls of ahakv_evict (for decode_round "
+                         "also --steps generation steps of each kind), nothing else")
     return ap.parse_args()
 
 
@@ -296,6 +297,25 @@ def run_ours(args):
     if args.capture:
         for i in range(args.steps):
             step(i)
+        if w.name == "decode_round":
+            # the generation step's kernels on the same cache, held at budget + 1 rows: the three-call step and the
+            # slot-cache step, --steps times each
+            Bud, n1 = w.budget, w.budget + 1
+            q, k, v = layers[0]
+            kc, vc = k[:, :, :n1].contiguous(), v[:, :, :n1].contiguous()
+            fc = torch.rand((w.batch, w.n_kv_heads, n1), device=dev)
+            idx1 = torch.empty((w.batch, w.n_kv_heads, Bud), dtype=torch.int32, device=dev)
+            pos = torch.arange(n1, dtype=torch.int32, device=dev).repeat(w.batch, w.n_kv_heads, 1).contiguous()
+            pos[:, :, Bud] = -1
+            free = torch.full((w.batch, w.n_kv_heads), Bud, dtype=torch.int32, device=dev)
+            for t in range(args.steps):
+                p1 = ab.Params(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, n1, 1, w.recent_window, Bud,
+                               dtype={"f32": ab.F32, "f16": ab.F16, "bf16": ab.BF16}[w.dtype], n_total=n1 + t, flags=0)
+                qt, kt, vt = synth.make_decode_step(w, t, device=dev)
+                ab.ahakv_score_step(p1, qt, kc, fc, fc, stream=stream)
+                ab.ahakv_select(p1, fc, idx1, stream=stream)
+                ab.ahakv_compact_inplace(p1, kc, vc, fc, idx1, stream=stream)
+                ab.ahakv_step_slots(p1, qt, kt, vt, kc, vc, fc, pos, free, stream=stream)
         barrier()
         print(json.dumps({"capture": True, "workload": w.name, "batch": w.batch, "steps": args.steps,
                           "warmup": n_warm, "device_status": ab.ahakv_last_device_status(ws)}))
