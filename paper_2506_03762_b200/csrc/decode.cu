@@ -30,22 +30,6 @@ constexpr size_t kStepMaxLogitBytes = 160 * 1024;   // 40960 logits
 
 template <typename T> using Acc = typename std::conditional<std::is_same<T, float>::value, double, float>::type;
 
-// Block-wide reduction in a fixed order: warp shuffles, then the warps' results in warp order.
-template <bool kMax>
-__device__ __forceinline__ float block_reduce(float x, float* red) {
-#pragma unroll
-  for (int o = 16; o; o >>= 1) {
-    const float y = __shfl_xor_sync(0xffffffffu, x, o);
-    x = kMax ? fmaxf(x, y) : x + y;
-  }
-  __syncthreads();                              // `red` may still be read from the last reduction
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
-  __syncthreads();
-  float r = red[0];
-  for (int w = 1; w < kStepThreads / 32; ++w) r = kMax ? fmaxf(r, red[w]) : r + red[w];
-  return r;
-}
-
 // The G x n logits of one (sequence, KV head), in log2 units, into shared memory.  LANES threads share a key row
 // (16 bytes each); kG query heads.
 template <typename T, int D, int kG>
@@ -188,33 +172,69 @@ __device__ __forceinline__ void step_logits_any(const T* __restrict__ q, const T
   else step_logits_mma<T, D, kG>(q, k, pl, b, h, (float)c_row, logit);
 }
 
-// Per query head: shift and normaliser, then 2^{x - M} / (G Z) in place of the logits.
-template <int kG>
-__device__ __forceinline__ void step_weights(float* logit, int n, float inv_g, float* red) {
+// kG block-wide reductions at once, each in a fixed order: warp shuffles, then the warps' results in warp order.
+template <bool kMax, int kG>
+__device__ __forceinline__ void block_reduce_heads(float (&x)[kG], float (*red)[kStepThreads / 32]) {
+#pragma unroll
   for (int g = 0; g < kG; ++g) {
-    float* x = logit + g * n;
-    float m = -INFINITY;
-    for (int j = threadIdx.x; j < n; j += kStepThreads) m = fmaxf(m, x[j]);
-    const float M = block_reduce<true>(m, red);
-    float z = 0.f;
-    for (int j = threadIdx.x; j < n; j += kStepThreads) {
-      const float e = fast_exp2(x[j] - M);
-      x[j] = e;
-      z += e;
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+      const float y = __shfl_xor_sync(0xffffffffu, x[g], o);
+      x[g] = kMax ? fmaxf(x[g], y) : x[g] + y;
     }
-    const float Z = block_reduce<false>(z, red);
-    const float w = inv_g / Z;
-    for (int j = threadIdx.x; j < n; j += kStepThreads) x[j] *= w;
+  }
+  __syncthreads();                              // `red` may still be read from the last reduction
+  if ((threadIdx.x & 31) == 0) {
+#pragma unroll
+    for (int g = 0; g < kG; ++g) red[g][threadIdx.x >> 5] = x[g];
   }
   __syncthreads();
+#pragma unroll
+  for (int g = 0; g < kG; ++g) {
+    float r = red[g][0];
+    for (int w = 1; w < kStepThreads / 32; ++w) r = kMax ? fmaxf(r, red[g][w]) : r + red[g][w];
+    x[g] = r;
+  }
+}
+
+// All query heads at once: shift and normaliser of every head, 2^{x - M} in place of the logits, and the factor
+// 1 / (G Z) of each head in w[].
+template <int kG>
+__device__ __forceinline__ void step_weights(float* logit, int n, float inv_g, float (*red)[kStepThreads / 32],
+                                             float (&w)[kG]) {
+  float m[kG];
+#pragma unroll
+  for (int g = 0; g < kG; ++g) m[g] = -INFINITY;
+  for (int j = threadIdx.x; j < n; j += kStepThreads) {
+#pragma unroll
+    for (int g = 0; g < kG; ++g) m[g] = fmaxf(m[g], logit[g * n + j]);
+  }
+  block_reduce_heads<true, kG>(m, red);
+  float z[kG];
+#pragma unroll
+  for (int g = 0; g < kG; ++g) z[g] = 0.f;
+  for (int j = threadIdx.x; j < n; j += kStepThreads) {
+#pragma unroll
+    for (int g = 0; g < kG; ++g) {
+      const float e = fast_exp2(logit[g * n + j] - m[g]);
+      logit[g * n + j] = e;                     // read back by the same thread only
+      z[g] += e;
+    }
+  }
+  block_reduce_heads<false, kG>(z, red);
+#pragma unroll
+  for (int g = 0; g < kG; ++g) w[g] = inv_g / z[g];
 }
 
 // Token j's share of the step: the weights of the group's heads pooled.
 template <int kG>
-__device__ __forceinline__ float step_pooled(const float* logit, int n, int j, int group_max) {
-  float s = logit[j];
+__device__ __forceinline__ float step_pooled(const float* logit, int n, int j, int group_max, const float (&w)[kG]) {
+  float s = logit[j] * w[0];
 #pragma unroll
-  for (int g = 1; g < kG; ++g) s = group_max ? fmaxf(s, logit[g * n + j]) : s + logit[g * n + j];
+  for (int g = 1; g < kG; ++g) {
+    const float t = logit[g * n + j] * w[g];
+    s = group_max ? fmaxf(s, t) : s + t;
+  }
   return s;
 }
 
@@ -224,12 +244,13 @@ __global__ void __launch_bounds__(kStepThreads) step_score_kernel(const T* __res
                                                                   float* __restrict__ score, const Shape pl,
                                                                   const double c_row) {
   extern __shared__ __align__(16) float logit[];                 // [kG][n]
-  __shared__ float red[kStepThreads / 32];
+  __shared__ float red[kG][kStepThreads / 32];
   const int unit = blockIdx.x, b = unit / pl.Hkv, h = unit % pl.Hkv, n = pl.n;
   step_logits_any<T, D, kG>(q, k, pl, b, h, c_row, logit);
-  step_weights<kG>(logit, n, pl.group_max ? 1.f : 1.f / (float)kG, red);
+  float w[kG];
+  step_weights<kG>(logit, n, pl.group_max ? 1.f : 1.f / (float)kG, red, w);
   for (int j = threadIdx.x; j < n; j += kStepThreads) {
-    float s = step_pooled<kG>(logit, n, j, pl.group_max);
+    float s = step_pooled<kG>(logit, n, j, pl.group_max, w);
     if (prev) s = __fadd_rn(s, prev[(size_t)unit * n + j]);
     score[(size_t)unit * n + j] = s;
   }
@@ -247,7 +268,7 @@ __global__ void __launch_bounds__(kStepThreads) step_slots_kernel(const T* __res
                                                                   int32_t* __restrict__ pos, int32_t* __restrict__ free_slot,
                                                                   const Shape pl, const double c_row, const int new_pos) {
   extern __shared__ __align__(16) float logit[];                 // [kG][n]
-  __shared__ float red[kStepThreads / 32];
+  __shared__ float red[kG][kStepThreads / 32];
   __shared__ unsigned long long best[kStepThreads / 32];
   constexpr int V = Vec16<T>::N, LANES = D / V;
   const int unit = blockIdx.x, b = unit / pl.Hkv, h = unit % pl.Hkv, n = pl.n;
@@ -266,12 +287,13 @@ __global__ void __launch_bounds__(kStepThreads) step_slots_kernel(const T* __res
   }
   __syncthreads();                                               // the row is read back by other threads below
   step_logits_any<T, D, kG>(q, k, pl, b, h, c_row, logit);
-  step_weights<kG>(logit, n, pl.group_max ? 1.f : 1.f / (float)kG, red);
+  float w[kG];
+  step_weights<kG>(logit, n, pl.group_max ? 1.f : 1.f / (float)kG, red, w);
   // F_t = SGsoftmax(A_t) + F_{t-1}, and the candidate to leave: smallest score, then largest position
   const int oldest_protected = new_pos - pl.Br + 1;             // positions from here on are the recent window
   unsigned long long mine = ~0ull;
   for (int j = threadIdx.x; j < n; j += kStepThreads) {
-    float s = step_pooled<kG>(logit, n, j, pl.group_max);
+    float s = step_pooled<kG>(logit, n, j, pl.group_max, w);
     const int pj = j == slot ? new_pos : ps[j];
     if (j != slot) s = __fadd_rn(s, sc[j]);                      // a new token starts at zero
     sc[j] = s;
