@@ -90,6 +90,25 @@ def test_bad_pointers_and_workspace_are_rejected_on_the_host(lib):
     assert ab.ahakv_workspace_bytes(_good(flags=ab.FLAG_GROUP_MAX)) > 0      # pooling by maximum is a legal request
 
 
+def test_the_generation_step_entry_points_reject_bad_requests_on_the_host(lib):
+    step = _good(n_ctx=257, obs_window=1, recent_window=16, budget=256, flags=0)
+    slots = lambda p=step, **kw: ab.ahakv_step_slots(p, kw.get("q", 256), kw.get("k_t", 256), kw.get("v_t", 256),
+                                                     kw.get("k", 256), kw.get("v", 256), kw.get("score", 256),
+                                                     kw.get("pos", 256), kw.get("free", 256), stream=0, check=False)
+    assert slots(q=None) == ab.ERR_INVALID_ARG
+    assert slots(k_t=8) == ab.ERR_INVALID_ARG             # not 16-byte aligned
+    assert slots(pos=None) == ab.ERR_INVALID_ARG
+    assert slots(free=2) == ab.ERR_INVALID_ARG            # not 4-byte aligned
+    # a slot cache holds budget + 1 rows and takes one query row
+    assert slots(_good(n_ctx=300, obs_window=1, recent_window=16, budget=256, flags=0)) == ab.ERR_INVALID_ARG
+    assert slots(_good(n_ctx=257, obs_window=2, recent_window=16, budget=256, flags=0)) == ab.ERR_INVALID_ARG
+    # the generation phase has no value prior
+    assert slots(_good(n_ctx=257, obs_window=1, recent_window=16, budget=256)) == ab.ERR_UNSUPPORTED
+    assert ab.ahakv_score_step(_good(n_ctx=257, obs_window=2, recent_window=16, budget=256, flags=0), 256, 256, None,
+                               256, stream=0, check=False) == ab.ERR_INVALID_ARG
+    assert ab.ahakv_compact_inplace(step, 256, None, None, 256, stream=0, check=False) == ab.ERR_INVALID_ARG
+
+
 def test_status_strings_and_errors(lib):
     assert ab.status_string(ab.OK) == "ok"
     assert "wait" in ab.status_string(ab.ERR_TIMEOUT)
