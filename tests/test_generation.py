@@ -260,3 +260,75 @@ def test_step_slots_for_48_steps(dtype_name, Hq, Hkv, d):
             for h in range(Hkv):
                 kept = np.array([j for j in range(n) if j != left[b, h]], dtype=np.int32)
                 parity.assert_kept_valid(p, kept, ref["kept_idx"][b, h], ref["score"][b, h])
+
+
+def test_step_slots_at_the_decode_shape():
+    """One step at the size the decode workload runs (16 sequences, 8 KV heads of 4 query heads, 2049 slots of 128,
+    bfloat16), slots in shuffled order: eight heads against the oracle on the cache in position order, and for every
+    head the bookkeeping (the slot that was free holds the new rows, one slot outside the recent window was freed,
+    every other position unchanged) and the invariant that the step adds exactly one unit of score per head."""
+    from paper_2506_03762_b200 import binding as ab
+    from tests import parity
+    w = synth.WORKLOADS["decode_round"]
+    B, Hq, Hkv, d, Bud, Br = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.budget, w.recent_window
+    n, N0 = Bud + 1, 40000
+    g = torch.Generator(device=DEV).manual_seed(31)
+    dt = torch.bfloat16
+    k = torch.randn((B, Hkv, n, d), device=DEV, generator=g).to(dt)
+    v = torch.randn((B, Hkv, n, d), device=DEV, generator=g).to(dt)
+    f = torch.rand((B, Hkv, n), device=DEV, generator=g) * 0.01
+    # positions: a random permutation of [N0 - n, N0 - 1) over the slots of each head, one slot free
+    perm = torch.argsort(torch.rand((B, Hkv, n), device=DEV, generator=g), dim=2)
+    pos = (perm + (N0 - n)).to(torch.int32)
+    free = (pos == N0 - 1).int().argmax(dim=2).to(torch.int32).contiguous()     # the slot "holding" position N0 - 1 is the free one
+    pos.scatter_(2, free.long()[:, :, None], torch.full((B, Hkv, 1), -1, dtype=torch.int32, device=DEV))
+    p = ab.Params(B, Hq, Hkv, d, n, 1, Br, Bud, dtype=ab.BF16, n_total=N0, flags=0)
+    new_pos = N0 - 1
+    q_t = torch.randn((B, Hq, 1, d), device=DEV, generator=g).to(dt)
+    k_t = torch.randn((B, Hkv, 1, d), device=DEV, generator=g).to(dt)
+    v_t = torch.randn((B, Hkv, 1, d), device=DEV, generator=g).to(dt)
+    k0, v0, f0, pos0, free0 = k.clone(), v.clone(), f.clone(), pos.clone(), free.clone()
+    ab.ahakv_step_slots(p, q_t, k_t, v_t, k, v, f, pos, free)
+    torch.cuda.synchronize()
+    fb, fa = free0.long()[:, :, None], free.long()[:, :, None]
+    pos_full = pos0.clone().scatter_(2, fb, torch.full_like(fb, new_pos, dtype=torch.int32))
+    k_full = k0.clone().scatter_(2, fb[..., None].expand(B, Hkv, 1, d), k_t)
+    v_full = v0.clone().scatter_(2, fb[..., None].expand(B, Hkv, 1, d), v_t)
+    assert torch.equal(k, k_full) and torch.equal(v, v_full)
+    assert torch.equal(pos, pos_full.clone().scatter_(2, fa, torch.full_like(fa, -1, dtype=torch.int32)))
+    assert bool((pos_full.gather(2, fa) < new_pos - Br + 1).all())
+    f_prev = f0.clone().scatter_(2, fb, torch.zeros_like(fb, dtype=torch.float32))
+    added = (f.double() - f_prev.double()).sum(dim=2)
+    assert float((added - 1.0).abs().max()) < 1e-3, "one query row per head, pooled by the mean: one unit of score a step"
+    order = torch.argsort(pos_full, dim=2)
+    rank_of_slot = torch.argsort(order, dim=2)
+    left = rank_of_slot.gather(2, fa)[:, :, 0].cpu().numpy()
+    for (b, h) in [(0, 0), (3, 5), (7, 2), (8, 7), (11, 1), (13, 4), (15, 7), (15, 0)]:
+        o = order[b, h]
+        op = parity.oracle_params(p, batch=1, n_q_heads=Hq // Hkv, n_kv_heads=1)
+        G = Hq // Hkv
+        ref = orc.evict(op, synth.to_numpy(q_t[b:b + 1, h * G:(h + 1) * G]), synth.to_numpy(k_full[b:b + 1, h:h + 1][:, :, o]),
+                        synth.to_numpy(v_full[b:b + 1, h:h + 1][:, :, o]), f_prev[b:b + 1, h:h + 1][:, :, o].double().cpu().numpy())
+        parity.assert_scores_close(p, f[b, h][o].cpu().numpy(), ref["score"][0, 0], f"unit ({b},{h})")
+        kept = np.array([j for j in range(n) if j != left[b, h]], dtype=np.int32)
+        parity.assert_kept_valid(p, kept, ref["kept_idx"][0, 0], ref["score"][0, 0])
+
+
+def test_score_step_at_its_largest_size():
+    """The most logits the one-row kernel takes (G n = 40960, all of a CTA's shared memory budget for them): four
+    heads a group against 10240 keys, checked against the oracle."""
+    from paper_2506_03762_b200 import binding as ab
+    from tests import parity
+    B, Hq, Hkv, d, n = 1, 8, 2, 128, 10240
+    g = torch.Generator().manual_seed(4096)
+    q = torch.randn((B, Hq, 1, d), generator=g).to(torch.float16).to(DEV)
+    k = torch.randn((B, Hkv, n, d), generator=g).to(torch.float16).to(DEV)
+    prev = (torch.rand((B, Hkv, n), generator=g) * 0.01).to(DEV)
+    p = ab.Params(B, Hq, Hkv, d, n, 1, 64, 4096, dtype=ab.F16, n_total=50000, flags=0)
+    got = torch.empty((B, Hkv, n), dtype=torch.float32, device=DEV)
+    ab.ahakv_score_step(p, q, k, prev, got)
+    ref = orc.score(parity.oracle_params(p), synth.to_numpy(q), synth.to_numpy(k), synth.to_numpy(k), prev.double().cpu().numpy())
+    parity.assert_scores_close(p, got.cpu().numpy(), ref, "score_step, 40960 logits")
+    # one more key is one too many
+    p2 = ab.Params(B, Hq, Hkv, d, n + 1, 1, 64, 4096, dtype=ab.F16, n_total=50000, flags=0)
+    assert ab.ahakv_score_step(p2, q, k, prev, got, check=False) == ab.ERR_UNSUPPORTED
