@@ -42,6 +42,8 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling small cases)")
+    ap.add_argument("--widened", action="store_true",
+                    help="time the entry points beyond the eviction step (variants, ragged batch, entropy) instead")
     ap.add_argument("--capture", action="store_true",
                     help="profiler-friendly run: exactly --warmup and --steps calls of ahakv_evict (for decode_round "
                          "also --steps generation steps of each kind), nothing else")
@@ -585,10 +587,88 @@ def decode_protocol(ab, synth, w, dev, stream):
     }
 
 
+def run_widened(args):
+    """Device times (CUDA events, median of 9 after 3 warm-ups) of the entry points beyond the eviction step, on
+    synthetic inputs of the long-context shape cut to what each call is for.  One JSON line."""
+    import statistics
+    import torch
+    from paper_2506_03762_b200 import binding as ab, synth
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ms = []
+        for _ in range(9):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream); fn(); e1.record(stream); torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+        return statistics.median(ms)
+
+    out = {"widened": True, "data": "synthetic", "timing": "CUDA events, median of 9 calls after 3"}
+    base = synth.WORKLOADS["long_32k"]
+
+    # accumulation over every causal row (Eq. 2-3) at 8192 tokens: 64 passes of 128 rows
+    w = base.scaled(batch=1, n_ctx=8192)
+    q, k, v = synth.make_layer(w, layer=0, device=dev)
+    q_all = torch.randn((w.batch, w.n_q_heads, w.n_ctx, w.head_dim), device=dev).to(k.dtype)
+    p = ab.Params(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.n_ctx, w.obs_window, w.recent_window, w.budget,
+                  dtype=ab.F16, flags=ab.FLAG_VALUE_PRIOR)
+    ws = ab.alloc_workspace(p, dev)
+    score = torch.empty((w.batch, w.n_kv_heads, w.n_ctx), dtype=torch.float32, device=dev)
+    ms = timed(lambda: ab.ahakv_score_full_causal(p, q_all, k, v, None, score, ws, stream=stream))
+    flops = 2.0 * w.batch * w.n_q_heads * w.head_dim * w.n_ctx * (w.n_ctx + 1) / 2 * 2     # two products, causal half
+    out["score_full_causal"] = {"shape": f"1 x {w.n_q_heads} heads x {w.n_ctx} tokens, all rows", "ms": ms,
+                                "passes": w.n_ctx // w.obs_window, "tflops_of_the_unmasked_part": flops / ms * 1e-9}
+    del q_all
+
+    # observation rows at scattered positions (the same kernels as ahakv_score)
+    w = base.scaled(batch=2)
+    q, k, v = synth.make_layer(w, layer=0, device=dev)
+    p = ab.Params(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.n_ctx, w.obs_window, w.recent_window, w.budget,
+                  dtype=ab.F16, flags=ab.FLAG_VALUE_PRIOR)
+    ws = ab.alloc_workspace(p, dev)
+    score = torch.empty((w.batch, w.n_kv_heads, w.n_ctx), dtype=torch.float32, device=dev)
+    rows = sorted(range(w.n_ctx - 1, w.n_ctx - 1 - 256 * w.obs_window, -256))
+    ms_rows = timed(lambda: ab.ahakv_score_rows(p, rows, q, k, v, None, score, ws, stream=stream))
+    ms_plain = timed(lambda: ab.ahakv_score(p, q, k, v, None, score, ws, stream=stream))
+    out["score_rows"] = {"shape": f"2 x {w.n_kv_heads} heads x {w.n_ctx} tokens, {w.obs_window} rows 256 apart", "ms": ms_rows,
+                         "ahakv_score_same_shape_ms": ms_plain}
+    # entropy of the observation rows (Eq. 6)
+    ent = torch.empty((w.batch, w.n_q_heads, w.obs_window), dtype=torch.float32, device=dev)
+    ms = timed(lambda: ab.ahakv_row_entropy(p, q, k, ent, stream=stream))
+    kbytes = k.numel() * k.element_size()
+    out["row_entropy"] = {"shape": out["score_rows"]["shape"].split(",")[0] + f", {w.obs_window} rows", "ms": ms,
+                          "gbs_of_k": kbytes / ms * 1e-6}
+
+    # a ragged batch: eight sequences of 2K .. 32K tokens, budgets a quarter of each
+    lens = [2048, 4096, 6144, 8192, 12288, 16384, 24576, 32768]
+    w = base.scaled(batch=len(lens))
+    q, k, v = synth.make_layer(w, layer=1, device=dev)
+    p = ab.Params(w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.n_ctx, w.obs_window, w.recent_window, w.n_ctx // 4,
+                  dtype=ab.F16, flags=ab.FLAG_VALUE_PRIOR)
+    ws = ab.alloc_workspace(p, dev)
+    k_out, v_out, s_out, idx = ab.alloc_outputs(p, dev)
+    seqs = [(n, n // 4, n) for n in lens]
+    ms = timed(lambda: ab.ahakv_evict_ragged(p, seqs, q, k, v, None, k_out, v_out, s_out, idx, ws, stream=stream))
+    assert ab.ahakv_last_device_status(ws) == ab.OK
+    tokens = sum(lens)
+    alg = sum(2 * n * w.n_kv_heads * w.head_dim * 2 for n in lens) + sum(4 * (n // 4) * w.n_kv_heads * w.head_dim * 2 for n in lens)
+    out["evict_ragged"] = {"shape": f"{len(lens)} sequences of {lens[0]} .. {lens[-1]} tokens, {w.n_kv_heads} heads", "ms": ms,
+                           "tokens_per_s": tokens / ms * 1e3, "gbs_algorithmic": alg / ms * 1e-6,
+                           "launch_sets": len(lens)}
+    print(json.dumps(out))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.widened:
+        run_widened(args)
     else:
         run_ours(args)
 

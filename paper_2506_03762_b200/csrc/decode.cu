@@ -19,6 +19,7 @@
 #include <type_traits>
 
 #include "ahakv_internal.cuh"
+#include "mma_sync.cuh"
 #include "select_common.cuh"
 
 namespace ahakv {
@@ -83,22 +84,6 @@ __device__ __forceinline__ void step_logits(const T* __restrict__ q, const T* __
 // thread takes one contiguous quarter of a row -- of its query head's row for the A operand, of its key's row for the
 // B operand -- and hands its 32-bit words to the instruction in pairs: the k-slices the four threads of a group
 // present side by side are then the same permutation of d for A and for B.
-template <typename T> struct Mma16816;
-template <> struct Mma16816<__half> {
-  static __device__ __forceinline__ void run(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                             uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-  }
-};
-template <> struct Mma16816<__nv_bfloat16> {
-  static __device__ __forceinline__ void run(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                             uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-  }
-};
-
 template <typename T, int D, int kG>
 __device__ __forceinline__ void step_logits_mma(const T* __restrict__ q, const T* __restrict__ k, const Shape& pl, int b,
                                                 int h, float c, float* logit) {

@@ -15,6 +15,7 @@ pytestmark = pytest.mark.gpu
     (1, 4, 4, 128, 4096, 64, "F16", {}),
     (1, 1, 1, 128, 300, 200, "F16", dict(scale_mode=0, scale=128 ** -0.5)),     # plain softmax, rows deep in the mask
     (1, 2, 1, 64, 129, 1, "BF16", {}),
+    (1, 2, 2, 64, 700, 256, "F16", {}),                                         # the most rows a call takes
 ])
 def test_row_entropy_matches_the_oracle(B, Hq, Hkv, d, n, r, dtype_name, extra):
     from paper_2506_03762_b200 import binding as ab
