@@ -191,6 +191,19 @@ ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k
                          const float* score_prev, void* k_out, void* v_out, float* score_out,
                          int32_t* kept_idx, void* ws, size_t ws_bytes, ahakv_stream_t stream);
 
+/* ahakv_evict with a budget of its own for every (sequence, KV head) (Algorithm 1 runs per head; the paper gives
+ * every head the same budget, allocators that do not can say so here).  head_budget: [B,Hkv] int32 in device
+ * memory, read by the selection kernel; an entry is held to [max(recent_window, 1), p->budget].  Head (b, h) keeps
+ * its recent window and the best head_budget[b,h] - recent_window of the rest.  Outputs keep the strides of
+ * ahakv_evict (n_keep = min(n_ctx, p->budget) rows a head): a head that keeps fewer fills kept_idx[b,h,t] with -1 from
+ * its own count on, and the rows of k_out, v_out and score_out from there on are left as they were.  The scores are
+ * those of ahakv_evict: in particular the scale of Eq. 12 is the call's, from p->budget, not one per head.  Tie
+ * rule and errors are ahakv_evict's too. */
+ahakv_status ahakv_evict_head_budgets(const ahakv_params* p, const int32_t* head_budget, const void* q_obs,
+                                      const void* k, const void* v, const float* score_prev, void* k_out, void* v_out,
+                                      float* score_out, int32_t* kept_idx, void* ws, size_t ws_bytes,
+                                      ahakv_stream_t stream);
+
 /* The whole step for a batch whose sequences differ in length, position and budget (a serving batch).  `p`
  * describes the allocation: p->n_ctx is the token extent of k, v and score_prev (the longest sequence's room),
  * p->budget the largest budget; everything else holds for all sequences.  seqs: HOST array of p->batch entries;

@@ -98,6 +98,7 @@ SIGNATURES = {
     "ahakv_select": (ctypes.c_int, [_PP, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_compact": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_evict": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "ahakv_evict_head_budgets": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_evict_ragged": (ctypes.c_int, [_PP, ctypes.POINTER(CSeq), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "ahakv_score_static": (ctypes.c_int, [_PP, _vp, _vp, _vp, _vp, _vp, _vp]),
     "ahakv_static_workspace_bytes": (_sz, []),
@@ -291,6 +292,19 @@ def ahakv_evict(p: Params, q_obs, k, v, score_prev, k_out, v_out, score_out, kep
                            _ptr(v_out), _ptr(score_out), _ptr(kept_idx), _ptr(ws), nbytes, _stream(stream))
     if check:
         _raise(st, "ahakv_evict")
+    return st
+
+
+def ahakv_evict_head_budgets(p: Params, head_budget, q_obs, k, v, score_prev, k_out, v_out, score_out, kept_idx, ws,
+                             ws_bytes: int | None = None, stream=None, check: bool = True) -> int:
+    """``ahakv_evict`` with ``head_budget`` [B,Hkv] int32 on the device: a budget per (sequence, KV head)."""
+    cp = p.c()
+    nbytes = ws.numel() * ws.element_size() if ws_bytes is None else ws_bytes
+    st = lib().ahakv_evict_head_budgets(ctypes.byref(cp), _ptr(head_budget), _ptr(q_obs), _ptr(k), _ptr(v),
+                                        _ptr(score_prev), _ptr(k_out), _ptr(v_out), _ptr(score_out), _ptr(kept_idx),
+                                        _ptr(ws), nbytes, _stream(stream))
+    if check:
+        _raise(st, "ahakv_evict_head_budgets")
     return st
 
 

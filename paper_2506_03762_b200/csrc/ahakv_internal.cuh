@@ -73,10 +73,12 @@ ahakv_status launch_vnorm(const Plan& pl, const void* v, float* nu, cudaStream_t
 // `slots` partial scores per head (row blocks, or query heads when pooling by maximum) are combined here.
 ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
                            float* score, int slots, cudaStream_t st);
-ahakv_status launch_select(const Plan& pl, const float* score, int32_t* kept_idx, cudaStream_t st);
+ahakv_status launch_select(const Plan& pl, const float* score, int32_t* kept_idx, const int32_t* budgets,
+                           cudaStream_t st);
 bool refine_select_fits(const Plan& pl);
 ahakv_status launch_refine_select(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
-                                  float* score, int32_t* kept_idx, int slots, cudaStream_t st);
+                                  float* score, int32_t* kept_idx, int slots, const int32_t* budgets,
+                                  cudaStream_t st);
 ahakv_status launch_compact(const Plan& pl, const void* k, const void* v, const float* score,
                             const int32_t* kept_idx, void* k_out, void* v_out, float* score_out,
                             cudaStream_t st);

@@ -329,7 +329,7 @@ ahakv_status ahakv_select(const ahakv_params* p, const float* score, int32_t* ke
   if (rc) return rc;
   if (!score || !kept_idx || !aligned16(score) || ((uintptr_t)kept_idx & 3)) return AHAKV_ERR_INVALID_ARG;
   (void)ws; (void)ws_bytes;                    // selection works in shared memory: no scratch is needed
-  return launch_select(pl, score, kept_idx, (cudaStream_t)stream);
+  return launch_select(pl, score, kept_idx, nullptr, (cudaStream_t)stream);
 }
 
 ahakv_status ahakv_compact(const ahakv_params* p, const void* k, const void* v, const float* score,
@@ -345,9 +345,9 @@ ahakv_status ahakv_compact(const ahakv_params* p, const void* k, const void* v, 
   return launch_compact(pl, k, v, score, kept_idx, k_out, v_out, score_out, (cudaStream_t)stream);
 }
 
-ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
-                         const float* score_prev, void* k_out, void* v_out, float* score_out,
-                         int32_t* kept_idx, void* ws, size_t ws_bytes, ahakv_stream_t stream) {
+static ahakv_status evict_impl(const ahakv_params* p, const int32_t* budgets, const void* q_obs, const void* k,
+                               const void* v, const float* score_prev, void* k_out, void* v_out, float* score_out,
+                               int32_t* kept_idx, void* ws, size_t ws_bytes, ahakv_stream_t stream) {
   Plan pl;
   ahakv_status rc = make_plan(p, &pl);
   if (rc) return rc;
@@ -364,17 +364,31 @@ ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k
   float* nu = prior ? at<float>(ws, pl.off_nu) : nullptr;
   float* score = at<float>(ws, pl.off_score);
   if (refine_select_fits(pl)) {      // a head's scores fit in one CTA's registers: both steps in one launch
-    rc = launch_refine_select(pl, s_raw, nu, score_prev, score, kept_idx, score_slots(pl), st);
+    rc = launch_refine_select(pl, s_raw, nu, score_prev, score, kept_idx, score_slots(pl), budgets, st);
     profile_mark(prof, 3, st);
   } else {
     rc = launch_refine(pl, s_raw, nu, score_prev, score, score_slots(pl), st);
     profile_mark(prof, 3, st);
-    if (rc == AHAKV_OK) rc = launch_select(pl, score, kept_idx, st);
+    if (rc == AHAKV_OK) rc = launch_select(pl, score, kept_idx, budgets, st);
   }
   profile_mark(prof, 4, st);
   if (rc == AHAKV_OK) rc = launch_compact(pl, k, v, score_out ? score : nullptr, kept_idx, k_out, v_out, score_out, st);
   profile_mark(prof, 5, st);
   return rc;
+}
+
+ahakv_status ahakv_evict(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
+                         const float* score_prev, void* k_out, void* v_out, float* score_out,
+                         int32_t* kept_idx, void* ws, size_t ws_bytes, ahakv_stream_t stream) {
+  return evict_impl(p, nullptr, q_obs, k, v, score_prev, k_out, v_out, score_out, kept_idx, ws, ws_bytes, stream);
+}
+
+ahakv_status ahakv_evict_head_budgets(const ahakv_params* p, const int32_t* head_budget, const void* q_obs, const void* k,
+                                      const void* v, const float* score_prev, void* k_out, void* v_out,
+                                      float* score_out, int32_t* kept_idx, void* ws, size_t ws_bytes,
+                                      ahakv_stream_t stream) {
+  if (!head_budget || ((uintptr_t)head_budget & 3)) return AHAKV_ERR_INVALID_ARG;
+  return evict_impl(p, head_budget, q_obs, k, v, score_prev, k_out, v_out, score_out, kept_idx, ws, ws_bytes, stream);
 }
 
 ahakv_status ahakv_evict_ragged(const ahakv_params* p, const ahakv_seq* seqs, const void* q_obs, const void* k,

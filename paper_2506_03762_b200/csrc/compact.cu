@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(const char* __restric
     const long long unit = row / pl.n_keep;
     const long long b = unit / pl.Hkv, h = unit % pl.Hkv;
     const int j = kept[row];
+    if (j < 0) continue;                       // a head with a budget of its own keeps fewer rows than the stride
     const long long ksrc = (b * pl.ks[0] + h * pl.ks[1] + (long long)j * pl.ks[2]) * pl.es + lane * 16;
     const long long vsrc = (b * pl.vs[0] + h * pl.vs[1] + (long long)j * pl.vs[2]) * pl.es + lane * 16;
     const long long dst = row * (long long)(LANES * 16) + lane * 16;

@@ -80,8 +80,18 @@ __device__ __forceinline__ void find_digit(const unsigned (*hist)[256], unsigned
   __syncthreads();
 }
 
+// The budget of one (sequence, KV head): the call's, or the caller's own for this head, held to [max(Br, 1), Bud].
+__device__ __forceinline__ int head_budget(const Shape& pl, const int32_t* budgets, int unit) {
+  if (budgets == nullptr) return pl.Bud;
+  return min(max(budgets[unit], max(pl.Br, 1)), pl.Bud);
+}
+// Entries of a head's index row beyond the tokens it keeps (heads with a budget of their own only).
+__device__ __forceinline__ void pad_kept(int32_t* out, int kept_here, int n_keep) {
+  for (int t = kept_here + threadIdx.x; t < n_keep; t += kThreads) out[t] = -1;
+}
+
 __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restrict__ score, int32_t* __restrict__ kept,
-                                                          const Shape pl) {
+                                                          const Shape pl, const int32_t* __restrict__ budgets) {
   __shared__ unsigned hist[1][256];
   __shared__ unsigned sh_prefix, sh_need, scan_tot[8];
   __shared__ int warp_gt[kWarps], warp_eq[kWarps];
@@ -89,11 +99,13 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const float* __restric
   const int unit = blockIdx.x, n = pl.n;
   const float* s = score + (size_t)unit * n;
   int32_t* out = kept + (size_t)unit * pl.n_keep;
-  if (n <= pl.Bud) {                       // nothing to evict
+  const int bud = head_budget(pl, budgets, unit);
+  pad_kept(out, min(n, bud), pl.n_keep);
+  if (n <= bud) {                          // nothing to evict
     for (int j = threadIdx.x; j < n; j += kThreads) out[j] = j;
     return;
   }
-  const int n_cand = n - pl.Br, Bs = pl.Bs;
+  const int n_cand = n - pl.Br, Bs = bud - pl.Br;
   for (int t = threadIdx.x; t < pl.Br; t += kThreads) out[Bs + t] = n_cand + t;   // recent window
   if (Bs == 0) return;
 
@@ -159,7 +171,8 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
                                                                     const float* __restrict__ nu,
                                                                     const float* __restrict__ prev,
                                                                     float* __restrict__ score, int32_t* __restrict__ kept,
-                                                                    const Shape pl, const int slots) {
+                                                                    const Shape pl, const int slots,
+                                                                    const int32_t* __restrict__ budgets) {
   __shared__ float red[kWarps];
   // four copies of the histogram, one per quarter of the warps: in the first passes nearly all keys of a head fall
   // into one or two bins, and the atomics on one counter are served one after the other
@@ -234,13 +247,15 @@ __global__ void __launch_bounds__(kThreads, 1) refine_select_kernel(const float*
   }
 
   int32_t* out = kept + (size_t)unit * pl.n_keep;
-  if (n <= pl.Bud) {                       // nothing to evict
+  const int bud = head_budget(pl, budgets, unit);
+  pad_kept(out, min(n, bud), pl.n_keep);
+  if (n <= bud) {                          // nothing to evict
 #pragma unroll
     for (int e = 0; e < kPer; ++e)
       if (e * kThreads + threadIdx.x < n) out[e * kThreads + threadIdx.x] = e * kThreads + threadIdx.x;
     return;
   }
-  const int n_cand = n - pl.Br, Bs = pl.Bs;
+  const int n_cand = n - pl.Br, Bs = bud - pl.Br;
   for (int t = threadIdx.x; t < pl.Br; t += kThreads) out[Bs + t] = n_cand + t;   // recent window
   if (Bs == 0) return;
 
@@ -328,8 +343,9 @@ ahakv_status launch_refine(const Plan& pl, const float* s_raw, const float* nu, 
   return cuda_ok(cudaGetLastError());
 }
 
-ahakv_status launch_select(const Plan& pl, const float* score, int32_t* kept_idx, cudaStream_t st) {
-  select_kernel<<<pl.B * pl.Hkv, kThreads, 0, st>>>(score, kept_idx, pl);
+ahakv_status launch_select(const Plan& pl, const float* score, int32_t* kept_idx, const int32_t* budgets,
+                           cudaStream_t st) {
+  select_kernel<<<pl.B * pl.Hkv, kThreads, 0, st>>>(score, kept_idx, pl, budgets);
   count_launch();
   return cuda_ok(cudaGetLastError());
 }
@@ -341,7 +357,8 @@ bool refine_select_fits(const Plan& pl) { return pl.n <= kPerMax * kThreads; }
 namespace {
 template <int kPer, bool kPrev>
 ahakv_status launch_refine_select_as(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
-                                     float* score, int32_t* kept_idx, int slots, cudaStream_t st) {
+                                     float* score, int32_t* kept_idx, int slots, const int32_t* budgets,
+                                     cudaStream_t st) {
   // Static and dynamic shared memory together may pass 48 KB well before the dynamic part alone does, and
   // beyond that the launch needs leave, asked for once per device: ask whenever the value norms are staged.
   constexpr int kMaxDevices = 64;
@@ -358,25 +375,26 @@ ahakv_status launch_refine_select_as(const Plan& pl, const float* s_raw, const f
     }
   }
   refine_select_kernel<kPer, kPrev><<<pl.B * pl.Hkv, kThreads, smem, st>>>(s_raw, nu, score_prev, score, kept_idx, pl,
-                                                                    slots);
+                                                                    slots, budgets);
   count_launch();
   return cuda_ok(cudaGetLastError());
 }
 }  // namespace
 
 ahakv_status launch_refine_select(const Plan& pl, const float* s_raw, const float* nu, const float* score_prev,
-                                  float* score, int32_t* kept_idx, int slots, cudaStream_t st) {
+                                  float* score, int32_t* kept_idx, int slots, const int32_t* budgets,
+                                  cudaStream_t st) {
   const int per = (pl.n + kThreads - 1) / kThreads;          // tokens a thread owns
   if (score_prev) {
-    if (per <= 4) return launch_refine_select_as<4, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
-    if (per <= 8) return launch_refine_select_as<8, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
-    if (per <= 16) return launch_refine_select_as<16, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
-    return launch_refine_select_as<kPerMax, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
+    if (per <= 4) return launch_refine_select_as<4, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, budgets, st);
+    if (per <= 8) return launch_refine_select_as<8, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, budgets, st);
+    if (per <= 16) return launch_refine_select_as<16, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, budgets, st);
+    return launch_refine_select_as<kPerMax, true>(pl, s_raw, nu, score_prev, score, kept_idx, slots, budgets, st);
   }
-  if (per <= 4) return launch_refine_select_as<4, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
-  if (per <= 8) return launch_refine_select_as<8, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
-  if (per <= 16) return launch_refine_select_as<16, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
-  return launch_refine_select_as<kPerMax, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, st);
+  if (per <= 4) return launch_refine_select_as<4, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, budgets, st);
+  if (per <= 8) return launch_refine_select_as<8, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, budgets, st);
+  if (per <= 16) return launch_refine_select_as<16, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, budgets, st);
+  return launch_refine_select_as<kPerMax, false>(pl, s_raw, nu, score_prev, score, kept_idx, slots, budgets, st);
 }
 
 }  // namespace ahakv
