@@ -4,7 +4,20 @@
 #include <cmath>
 #include <cstring>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "ahakv_internal.cuh"
+
+// A named range on the host's timeline for a profiler's trace (NVTX; costs nothing when no tool is attached): one
+// around every eviction call and one around the launches of each of its phases.
+namespace {
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
+}  // namespace
 
 static_assert(sizeof(ahakv_params) == 136, "ahakv_params layout is part of the ABI");
 
@@ -133,6 +146,7 @@ template <typename T> static T* at(void* ws, size_t off) { return reinterpret_ca
 // norms in the workspace.
 static ahakv_status queue_raw_score(const Plan& pl, const void* q, const void* k, const void* v, void* ws,
                                     cudaStream_t st, int prof) {
+  TraceRange range("ahakv: score");
   ahakv_status rc = cuda_ok(cudaMemsetAsync(at<char>(ws, pl.off_status), 0, pl.off_sraw - pl.off_status, st));
   if (rc) return rc;
   profile_mark(prof, 0, st);
@@ -357,12 +371,14 @@ static ahakv_status evict_impl(const ahakv_params* p, const int32_t* budgets, co
     return AHAKV_ERR_INVALID_ARG;
   if ((rc = check_ws(pl, ws, ws_bytes))) return rc;
   cudaStream_t st = (cudaStream_t)stream;
+  TraceRange call("ahakv_evict");
   const int prof = profile_begin_call(st);
   if ((rc = queue_raw_score(pl, q_obs, k, v, ws, st, prof))) return rc;
   const bool prior = (pl.flags & AHAKV_FLAG_VALUE_PRIOR) != 0;
   float* s_raw = at<float>(ws, pl.off_sraw);
   float* nu = prior ? at<float>(ws, pl.off_nu) : nullptr;
   float* score = at<float>(ws, pl.off_score);
+  nvtxRangePushA("ahakv: refine + select");
   if (refine_select_fits(pl)) {      // a head's scores fit in one CTA's registers: both steps in one launch
     rc = launch_refine_select(pl, s_raw, nu, score_prev, score, kept_idx, score_slots(pl), budgets, st);
     profile_mark(prof, 3, st);
@@ -371,8 +387,12 @@ static ahakv_status evict_impl(const ahakv_params* p, const int32_t* budgets, co
     profile_mark(prof, 3, st);
     if (rc == AHAKV_OK) rc = launch_select(pl, score, kept_idx, budgets, st);
   }
+  nvtxRangePop();
   profile_mark(prof, 4, st);
-  if (rc == AHAKV_OK) rc = launch_compact(pl, k, v, score_out ? score : nullptr, kept_idx, k_out, v_out, score_out, st);
+  {
+    TraceRange range("ahakv: compact");
+    if (rc == AHAKV_OK) rc = launch_compact(pl, k, v, score_out ? score : nullptr, kept_idx, k_out, v_out, score_out, st);
+  }
   profile_mark(prof, 5, st);
   return rc;
 }
