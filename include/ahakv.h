@@ -93,7 +93,12 @@ double ahakv_lambda(int64_t n_total, int32_t budget, int32_t head_dim);
  *   with score_prev != NULL: S_j += score_prev_j (Algorithm 1: F_t = ... + F_{t-1}).
  * Observation row i sits at logical position n_total - r + i and sees cache rows 0 .. n - r + i.
  * score_prev: nullable, [B,Hkv,n] float32.  score: [B,Hkv,n] float32 out.
- * v may be NULL when the value prior is off. */
+ * v may be NULL when the value prior is off.
+ * Resources: for 16-bit inputs and n_ctx >= 128 the scoring kernel is launched cooperatively with one CTA per SM
+ * and takes each SM's whole tensor memory (512 columns) and nearly all of its shared memory for its duration.  A
+ * kernel of the caller's that allocates tensor memory and runs concurrently on another stream can be held up
+ * until it ends, and holds it up the same way: the allocation is the hardware's, and the time it waits does not
+ * count against the kernel's own bounded waits.  Do not overlap such kernels with this call. */
 ahakv_status ahakv_score(const ahakv_params* p, const void* q_obs, const void* k, const void* v,
                          const float* score_prev, float* score, void* ws, size_t ws_bytes,
                          ahakv_stream_t stream);
