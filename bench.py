@@ -356,6 +356,30 @@ def run_ours(args):
     warm_ms_step = max_over_ranks(w0.elapsed_time(w1), world, dev) / args.steps
     tokens_per_step = w.batch * w.n_ctx
     value = whole_job_value(tokens_per_step, world, ms_step)
+    # the same K steps captured once in a CUDA graph and replayed: what the call costs without the host's launch
+    # overhead (it matters for the small workloads, whose kernels are shorter than the gaps between them)
+    graph_ms_step = None
+    if world == 1:
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        outer = stream
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                stream = torch.cuda.current_stream()
+                for i in range(args.steps):
+                    step(i)
+        stream = outer
+        torch.cuda.synchronize()
+        reps = []
+        for _ in range(3):
+            w0.record(side)
+            with torch.cuda.stream(side):
+                graph.replay()
+            w1.record(side)
+            torch.cuda.synchronize()
+            reps.append(w0.elapsed_time(w1) / args.steps)
+        graph_ms_step = statistics.median(reps)
+        del graph
 
     # ---- per-stage device times over the same K steps (events inside the library) ----------------------
     ab.ahakv_profile_enable(True)
@@ -432,6 +456,7 @@ def run_ours(args):
         "path_roofline": {"t_roof_ms": t_roof_ms, "frac": t_roof_ms / ms_step, "algorithmic_bytes": work["bytes"],
                           "flops": work["flops"], "frac_vs_spec_8TBs": 1e3 * work["bytes"] / (SPEC_HBM_GBS * 1e9) / ms_step,
                           "of": pk["source"]},
+        "ms_per_step_replayed_from_a_cuda_graph": graph_ms_step,
         "stage_ms": stage_ms,
         "stage_gbs": {s: stage_bytes[s] / (stage_ms[s] * 1e-3) / 1e9 for s in stage_bytes if stage_ms.get(s, 0) > 0},
         "tokens_per_step": tokens_per_step,

@@ -305,3 +305,33 @@ def test_wrong_device_arguments_leave_outputs_untouched():
     torch.cuda.synchronize()
     assert (idx == -7).all()
     assert ab.ahakv_launch_count() >= 0
+
+
+def test_the_eviction_call_replays_from_a_cuda_graph():
+    """ahakv_evict (two memsets, the cooperative scoring kernel, selection, compaction) captured once and replayed:
+    the same kept indices, rows and scores as the eager call, and a clean device status."""
+    from paper_2506_03762_b200 import binding as ab
+    from tests import parity
+    B, Hq, Hkv, d, n, r, Br, Bud = 2, 8, 4, 128, 3000, 32, 32, 512
+    g = torch.Generator().manual_seed(99)
+    q = torch.randn((B, Hq, r, d), generator=g).to(torch.float16).cuda()
+    k = torch.randn((B, Hkv, n, d), generator=g).to(torch.float16).cuda()
+    v = torch.randn((B, Hkv, n, d), generator=g).to(torch.float16).cuda()
+    p = ab.Params(B, Hq, Hkv, d, n, r, Br, Bud, dtype=ab.F16)
+    eager = parity.run_evict(p, q, k, v, None)
+    ws = ab.alloc_workspace(p, "cuda")
+    outs = ab.alloc_outputs(p, "cuda")
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            ab.ahakv_evict(p, q, k, v, None, *outs, ws, stream=torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    for _ in range(2):
+        for t in outs:
+            t.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ab.ahakv_last_device_status(ws) == ab.OK
+        for a, c in zip(eager, outs):
+            assert torch.equal(a, c)
